@@ -1,0 +1,179 @@
+/*
+ * flowmm.h - C ABI of the FlowMM KV-cache compression library for NVIDIA B200 (sm_100a).
+ *
+ * FlowMM (arXiv 2511.05534, Section 3.3) compresses each transformer layer's KV cache once,
+ * after multimodal prefill, per KV head:
+ *   1. score   - attention of the proxy tokens (the last W prompt positions) over all context
+ *                keys gives every token an importance (Eq. 8); the same attention, split by
+ *                modality, gives the layer's cross-modal interaction ratio rho (Eq. 6-7);
+ *   2. flow    - rho against the threshold theta picks cross-modal or intra-modal merging;
+ *   3. select  - the B most important tokens form the pivot set, the rest the non-pivot set;
+ *   4. match   - each non-pivot finds the pivot of largest key cosine similarity (Eq. 9)
+ *                among pivots whose importance does not exceed the sensitivity threshold
+ *                tau (Eq. 10) and, in an intra-modal layer, that share its modality;
+ *   5. merge   - non-pivots are folded into their pivots (Eq. 5) and the B merged rows are
+ *                written out as the compressed cache.
+ *
+ * Conventions for every entry point
+ *   - A "unit" is one (layer, sequence) pair; units are independent problems and a call
+ *     processes n_units of them at once.  G = n_q_heads / n_kv_heads query heads share KV
+ *     head h = g / G.  L = seq_len, W = window, B = n_keep, E = L - B.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; the library allocates
+ *     and frees nothing.  Scratch memory comes from the caller as `ws` / `ws_bytes`
+ *     (size from flowmm_workspace_bytes, 256-byte aligned); its first word is a sticky
+ *     device status, so the caller zero-fills the first 256 bytes once after allocating
+ *     it.  Inputs are never written; outputs must not alias inputs.
+ *   - n_units * n_kv_heads must not exceed 65535 per call (a CUDA grid dimension).
+ *   - Q, K, V and the outputs have the element type `dtype`, head_dim contiguous, and the
+ *     element strides given in the params (unit, head, token).  Base pointers must be
+ *     16-byte aligned and every stride a multiple of 8 elements, else FLOWMM_ERR_ALIGN.
+ *     All other arrays are dense in the stated shape.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without waiting.  The return value reports host-side validation
+ *     and launch errors.  Problems found on the device (a bounded wait that ran out) set
+ *     the status word, which flowmm_last_device_status reads back.
+ *   - There is no CPU fallback: on a device that is not compute capability 10.x every
+ *     compute entry point returns FLOWMM_ERR_UNSUPPORTED_DEVICE.
+ */
+#ifndef FLOWMM_H_
+#define FLOWMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FLOWMM_OK = 0,
+    FLOWMM_ERR_NULL = 1,               /* a required pointer is NULL */
+    FLOWMM_ERR_SHAPE = 2,              /* sizes inconsistent (heads, head_dim, window, ...) */
+    FLOWMM_ERR_BUDGET = 3,             /* n_keep outside [1, L], or below W with keep_window */
+    FLOWMM_ERR_DTYPE = 4,
+    FLOWMM_ERR_WORKSPACE = 5,          /* ws_bytes smaller than flowmm_workspace_bytes */
+    FLOWMM_ERR_ALIGN = 6,
+    FLOWMM_ERR_CUDA = 7,               /* a CUDA runtime call or launch failed */
+    FLOWMM_ERR_TIMEOUT = 8,            /* device status: a bounded wait inside a kernel ran out */
+    FLOWMM_ERR_UNSUPPORTED_DEVICE = 9
+} flowmm_status;
+
+typedef enum { FLOWMM_F32 = 0, FLOWMM_BF16 = 1 } flowmm_dtype;
+typedef enum { FLOWMM_INTRA = 0, FLOWMM_CROSS = 1 } flowmm_strategy;
+/* Eq. 5 leaves the merge functions open.  EXPSIM: pivot weight 1, non-pivot weight
+ * exp(u - 1) with u its cosine similarity to the pivot; MEAN: all weights 1.  Weights are
+ * normalised to sum to one per output row. */
+typedef enum { FLOWMM_MERGE_EXPSIM = 0, FLOWMM_MERGE_MEAN = 1 } flowmm_merge_mode;
+/* ABS: tau is compared with the importance directly.  REL: tau is in units of the
+ * importance a uniform attention would give, tau_eff = tau * W / L. */
+typedef enum { FLOWMM_TAU_ABS = 0, FLOWMM_TAU_REL = 1 } flowmm_tau_mode;
+typedef enum { FLOWMM_FLOW_AUTO = 0, FLOWMM_FLOW_FORCE_INTRA = 1, FLOWMM_FLOW_FORCE_CROSS = 2 } flowmm_flow_mode;
+/* Which kernels do the two dense contractions.  AUTO: tensor-core (tcgen05) kernels when
+ * dtype is bf16 and head_dim is 128, SIMT fp32 kernels otherwise.  SIMT forces the latter. */
+typedef enum { FLOWMM_PATH_AUTO = 0, FLOWMM_PATH_SIMT = 1 } flowmm_path;
+
+typedef struct {
+    int32_t n_units;                    /* independent (layer, sequence) problems */
+    int32_t n_q_heads, n_kv_heads;      /* n_q_heads must be a multiple of n_kv_heads */
+    int32_t head_dim;                   /* 64 or 128 */
+    int32_t seq_len, window;            /* L, W with 1 <= W <= L */
+    int32_t n_keep;                     /* B with 1 <= B <= L */
+    int32_t dtype;                      /* flowmm_dtype of Q, K, V, K_out, V_out */
+    float softmax_scale;                /* 0 selects 1/sqrt(head_dim) */
+    float theta;                        /* cross-modal merging threshold of Section 3.3.1 */
+    float tau;                          /* sensitivity threshold of Eq. 10; +inf disables it */
+    int32_t tau_mode;                   /* flowmm_tau_mode */
+    int32_t flow_mode;                  /* flowmm_flow_mode */
+    int32_t merge_mode;                 /* flowmm_merge_mode */
+    int32_t keep_window;                /* 1: the W proxy tokens are always pivots (needs B >= W) */
+    int32_t path;                       /* flowmm_path */
+    /* element strides of (unit, head, token); head_dim stride is 1 */
+    int64_t q_stride[3];                /* Q_win [U, Hq,  W, D] */
+    int64_t k_stride[3];                /* K     [U, Hkv, L, D] */
+    int64_t v_stride[3];                /* V     [U, Hkv, L, D] */
+    int64_t ko_stride[3];               /* K_out [U, Hkv, B, D] */
+    int64_t vo_stride[3];               /* V_out [U, Hkv, B, D] */
+} flowmm_params;
+
+/* Scratch size in bytes that any entry point below needs for these params.  Host only; makes
+ * no CUDA call.  Fails with the same validation errors as the compute entry points. */
+flowmm_status flowmm_workspace_bytes(const flowmm_params *p, size_t *bytes);
+
+/*
+ * Step 1, Eq. 8 (with the causal softmax of Eq. 4 on the proxy rows) and the masses of Eq. 7.
+ *   q_win      [U, Hq, W, D]   queries of the last W prompt positions
+ *   k          [U, Hkv, L, D]  layer keys
+ *   modality   [U, L] uint8    0 = text token, 1 = visual token
+ *   importance [U, Hkv, L] f32 out: I[h,i] = (1/G) sum_{g in h} sum_a alpha[g,a,i]
+ *   cross_mass [U, Hq] f32     out: sum_a sum_{i: m_i != m_(p_a)} alpha[g,a,i]; the total mass
+ *                              of a head is W because every softmax row sums to one.
+ */
+flowmm_status flowmm_score(const flowmm_params *p, const void *q_win, const void *k, const uint8_t *modality,
+                           float *importance, float *cross_mass, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Step 2, Eq. 6 and the threshold rule after Eq. 7.
+ *   rho      [U] f32   out: mean over query heads of cross_mass / W
+ *   strategy [U] int32 out: FLOWMM_CROSS if rho > theta else FLOWMM_INTRA (or as flow_mode forces)
+ */
+flowmm_status flowmm_layer_flow(const flowmm_params *p, const float *cross_mass, float *rho, int32_t *strategy,
+                                void *cuda_stream);
+
+/*
+ * Step 3, pivot selection of Section 3.3.1: the B largest importances per KV head, ties to the
+ * lower index.
+ *   retained_idx [U, Hkv, B] int32 out: pivot token positions, ascending; slot s holds r_s
+ *   evicted_idx  [U, Hkv, E] int32 out: non-pivot token positions, ascending
+ */
+flowmm_status flowmm_select(const flowmm_params *p, const float *importance, int32_t *retained_idx,
+                            int32_t *evicted_idx, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Step 4, Eq. 9 and Eq. 10.  For the j-th non-pivot e = evicted_idx[j]:
+ *   match     [U, Hkv, E] int32 out: slot of the admissible pivot with the largest cosine
+ *                                    similarity (ties to the lower slot), or -1 if none
+ *   match_sim [U, Hkv, E] f32   out: that similarity, 0 where match is -1
+ * A pivot r_s is admissible if importance[r_s] <= tau_eff and, when strategy[u] is
+ * FLOWMM_INTRA, modality[r_s] == modality[e].  A key of zero norm has similarity 0.
+ */
+flowmm_status flowmm_match(const flowmm_params *p, const void *k, const float *importance, const uint8_t *modality,
+                           const int32_t *retained_idx, const int32_t *evicted_idx, const int32_t *strategy,
+                           int32_t *match, float *match_sim, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Step 5, Eq. 5 and compaction.  Output row s (s in [0, B), ascending token position) is
+ *   (x[r_s] + sum_{j: match[j] = s} w_j x[e_j]) / (1 + sum w_j),  x in {K, V},
+ * with w_j = exp(match_sim[j] - 1) (EXPSIM) or 1 (MEAN); non-pivots with match -1 are dropped.
+ * Accumulation is fp32 in a fixed order (results are bit-reproducible), rounded once to dtype.
+ *   k_out, v_out [U, Hkv, B, D]
+ */
+flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v, const int32_t *retained_idx,
+                           const int32_t *evicted_idx, const int32_t *match, const float *match_sim,
+                           void *k_out, void *v_out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Steps 1-5 in order on one stream: the whole per-layer FlowMM compression of Section 3.3.
+ * The diagnostic outputs (importance ... match_sim, layouts as above) may each be NULL, in
+ * which case the intermediate lives in the workspace only.
+ */
+flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, const void *k, const void *v,
+                                    const uint8_t *modality, void *k_out, void *v_out,
+                                    float *importance, float *rho, int32_t *strategy,
+                                    int32_t *retained_idx, int32_t *evicted_idx,
+                                    int32_t *match, float *match_sim,
+                                    void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Waits for `cuda_stream`, then returns the device status word at the start of `ws`
+ * (FLOWMM_OK, or the first error a kernel recorded) and clears it. */
+flowmm_status flowmm_last_device_status(void *ws, void *cuda_stream);
+
+/* Number of kernels the most recent compute entry point of this thread enqueued. */
+int32_t flowmm_last_launch_count(void);
+
+/* Static, human-readable name of a status code. */
+const char *flowmm_status_string(flowmm_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLOWMM_H_ */

@@ -1,0 +1,392 @@
+// C ABI of the FlowMM compression library: validation, workspace layout and kernel launches.
+// Declarations and the meaning of every argument are in include/flowmm.h.
+#include "flowmm.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "select_merge.cuh"
+#include "simt_kernels.cuh"
+
+using namespace flowmm;
+
+namespace {
+
+thread_local int32_t g_launches = 0;
+
+#define FLOWMM_LAUNCH_CHECK()                                   \
+    do {                                                        \
+        ++g_launches;                                           \
+        if (cudaGetLastError() != cudaSuccess) return FLOWMM_ERR_CUDA; \
+    } while (0)
+
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// Where everything lives inside the caller's workspace.  One layout serves every entry point.
+struct Layout {
+    size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
+    size_t row_part, cross_part, rn, sort_a, sort_b, off, piece_off, part_off, partial;
+    size_t total;
+    int n_chunk1, chunk1, n_chunk2, chunk2, max_pieces, max_parts, csr_passes;
+};
+
+int chunks_for(int L, int other_ctas, int &chunk) {
+    // enough CTAs to fill the GPU about twice, at least 64 keys per chunk
+    int want = (2 * 148 + other_ctas - 1) / other_ctas;
+    const int max_chunks = (L + kTile - 1) / kTile;
+    if (want < 1) want = 1;
+    if (want > max_chunks) want = max_chunks;
+    chunk = ((L + want - 1) / want + kTile - 1) / kTile * kTile;
+    return (L + chunk - 1) / chunk;
+}
+
+Layout make_layout(const flowmm_params &p) {
+    Layout y;
+    const size_t U = p.n_units, Hq = p.n_q_heads, Hkv = p.n_kv_heads, L = p.seq_len, W = p.window;
+    const size_t B = p.n_keep, E = L - B, D = p.head_dim, G = Hq / Hkv;
+    const int row_tiles = (int)((G * W + kTile - 1) / kTile);
+    y.n_chunk1 = chunks_for((int)L, (int)(U * Hkv) * row_tiles, y.chunk1);
+    y.n_chunk2 = chunks_for((int)L, (int)(U * Hkv), y.chunk2);
+    y.max_pieces = (int)(B + E / kPiece + 1);
+    y.max_parts = (int)(2 * (E / kPiece) + 2);
+    y.csr_passes = 1;
+    while (y.csr_passes < 4 && (B >> (8 * y.csr_passes)) != 0) ++y.csr_passes;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { const size_t at = o; o += align256(bytes); return at; };
+    y.status = take(256);
+    y.importance = take(U * Hkv * L * 4);
+    y.cross_mass = take(U * Hq * 4);
+    y.rho = take(U * 4);
+    y.strategy = take(U * 4);
+    y.retained = take(U * Hkv * B * 4);
+    y.evicted = take(U * Hkv * E * 4);
+    y.match = take(U * Hkv * E * 4);
+    y.match_sim = take(U * Hkv * E * 4);
+    y.row_part = take(U * Hq * W * (size_t)y.n_chunk1 * 8);
+    y.cross_part = take(U * Hq * (size_t)y.n_chunk2 * 4);
+    y.rn = take(U * Hkv * L * 4);
+    y.sort_a = take(U * Hkv * E * 4);
+    y.sort_b = take(U * Hkv * E * 4);
+    y.off = take(U * Hkv * (B + 1) * 4);
+    y.piece_off = take(U * Hkv * (B + 1) * 4);
+    y.part_off = take(U * Hkv * (B + 1) * 4);
+    y.partial = take(U * Hkv * (size_t)y.max_parts * (2 * D + 4) * 4);
+    y.total = o;
+    return y;
+}
+
+flowmm_status validate(const flowmm_params *p) {
+    if (!p) return FLOWMM_ERR_NULL;
+    if (p->n_units < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1) return FLOWMM_ERR_SHAPE;
+    if (p->n_q_heads % p->n_kv_heads != 0) return FLOWMM_ERR_SHAPE;
+    if (p->head_dim != 64 && p->head_dim != 128) return FLOWMM_ERR_SHAPE;
+    if (p->seq_len < 1 || p->window < 1 || p->window > p->seq_len) return FLOWMM_ERR_SHAPE;
+    if ((int64_t)p->n_units * p->n_kv_heads > 65535) return FLOWMM_ERR_SHAPE;
+    if (p->n_keep < 1 || p->n_keep > p->seq_len) return FLOWMM_ERR_BUDGET;
+    if (p->keep_window && p->n_keep < p->window) return FLOWMM_ERR_BUDGET;
+    if (p->dtype != FLOWMM_F32 && p->dtype != FLOWMM_BF16) return FLOWMM_ERR_DTYPE;
+    if (p->tau_mode < 0 || p->tau_mode > 1 || p->flow_mode < 0 || p->flow_mode > 2 || p->merge_mode < 0 ||
+        p->merge_mode > 1 || p->path < 0 || p->path > 1)
+        return FLOWMM_ERR_SHAPE;
+    if (!(p->softmax_scale >= 0.f) || isnan(p->theta) || isnan(p->tau)) return FLOWMM_ERR_SHAPE;
+    return FLOWMM_OK;
+}
+
+bool strides_ok(const int64_t s[3], int head_dim) {
+    for (int i = 0; i < 3; ++i)
+        if (s[i] < 0 || s[i] % 8 != 0) return false;
+    return s[2] >= head_dim;
+}
+bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }
+
+flowmm_status check_device() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    return major == 10 ? FLOWMM_OK : FLOWMM_ERR_UNSUPPORTED_DEVICE;
+}
+
+flowmm_status check_ws(const flowmm_params *p, const void *ws, size_t ws_bytes, Layout &y) {
+    if (!ws) return FLOWMM_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(ws) & 255) return FLOWMM_ERR_ALIGN;
+    y = make_layout(*p);
+    if (ws_bytes < y.total) return FLOWMM_ERR_WORKSPACE;
+    return FLOWMM_OK;
+}
+
+template <typename X> X *at(void *ws, size_t off) { return reinterpret_cast<X *>(static_cast<char *>(ws) + off); }
+
+float tau_effective(const flowmm_params &p) {
+    return p.tau_mode == FLOWMM_TAU_REL ? (float)((double)p.tau * (double)p.window / (double)p.seq_len) : p.tau;
+}
+
+// ---- step launchers (no validation; the entry points below validate) --------------------------
+
+flowmm_status run_score(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
+                        float *importance, float *cross_mass, void *ws, cudaStream_t st) {
+    ScoreArgs a;
+    a.q = q; a.k = k; a.modality = mod; a.importance = importance;
+    a.row_part = at<float2>(ws, y.row_part);
+    a.cross_part = at<float>(ws, y.cross_part);
+    a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.G = p.n_q_heads / p.n_kv_heads;
+    a.D = p.head_dim; a.L = p.seq_len; a.W = p.window;
+    a.n_chunk1 = y.n_chunk1; a.chunk1 = y.chunk1; a.n_chunk2 = y.n_chunk2; a.chunk2 = y.chunk2;
+    const float scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * kLog2e;
+    for (int i = 0; i < 3; ++i) { a.qs[i] = p.q_stride[i]; a.ks[i] = p.k_stride[i]; }
+    const int GW = a.G * a.W;
+    const int UH = p.n_units * p.n_kv_heads;
+    const dim3 g1(y.n_chunk1, (GW + kTile - 1) / kTile, UH), g2(y.n_chunk2, 1, UH);
+    const size_t dyn = (size_t)3 * GW * sizeof(float);
+    if (p.dtype == FLOWMM_BF16) {
+        score_stats_simt<__nv_bfloat16><<<g1, kSimtThreads, 0, st>>>(a);
+        FLOWMM_LAUNCH_CHECK();
+        score_colsum_simt<__nv_bfloat16><<<g2, kSimtThreads, dyn, st>>>(a);
+        FLOWMM_LAUNCH_CHECK();
+    } else {
+        score_stats_simt<float><<<g1, kSimtThreads, 0, st>>>(a);
+        FLOWMM_LAUNCH_CHECK();
+        score_colsum_simt<float><<<g2, kSimtThreads, dyn, st>>>(a);
+        FLOWMM_LAUNCH_CHECK();
+    }
+    const int n = p.n_units * p.n_q_heads;
+    cross_mass_reduce<<<(n + 255) / 256, 256, 0, st>>>(a.cross_part, y.n_chunk2, n, cross_mass);
+    FLOWMM_LAUNCH_CHECK();
+    return FLOWMM_OK;
+}
+
+flowmm_status run_layer_flow(const flowmm_params &p, const float *cross_mass, float *rho, int32_t *strategy,
+                             cudaStream_t st) {
+    layer_flow_kernel<<<(p.n_units + 127) / 128, 128, 0, st>>>(cross_mass, p.n_units, p.n_q_heads, p.window, p.theta,
+                                                                p.flow_mode, rho, strategy);
+    FLOWMM_LAUNCH_CHECK();
+    return FLOWMM_OK;
+}
+
+flowmm_status run_select(const flowmm_params &p, const float *importance, int32_t *retained, int32_t *evicted,
+                         cudaStream_t st) {
+    select_topb_kernel<<<p.n_units * p.n_kv_heads, kSelectThreads, 0, st>>>(importance, p.seq_len, p.n_keep, p.window,
+                                                                           p.keep_window, retained, evicted);
+    FLOWMM_LAUNCH_CHECK();
+    return FLOWMM_OK;
+}
+
+flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
+                        const uint8_t *mod, const int32_t *retained, const int32_t *evicted, const int32_t *strategy,
+                        int32_t *match, float *match_sim, void *ws, cudaStream_t st) {
+    const int E = p.seq_len - p.n_keep;
+    if (E == 0) return FLOWMM_OK;
+    float *rn = at<float>(ws, y.rn);
+    const int64_t rows = (int64_t)p.n_units * p.n_kv_heads * p.seq_len;
+    const int lanes = p.head_dim / (p.dtype == FLOWMM_BF16 ? 8 : 4);
+    const int64_t threads = rows * lanes;
+    const unsigned blocks = (unsigned)((threads + 255) / 256);
+    if (p.dtype == FLOWMM_BF16)
+        inv_norm_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(k, rows, p.n_kv_heads, p.seq_len, p.head_dim,
+                                                               p.k_stride[0], p.k_stride[1], p.k_stride[2], rn);
+    else
+        inv_norm_kernel<float><<<blocks, 256, 0, st>>>(k, rows, p.n_kv_heads, p.seq_len, p.head_dim, p.k_stride[0],
+                                                       p.k_stride[1], p.k_stride[2], rn);
+    FLOWMM_LAUNCH_CHECK();
+    MatchArgs a;
+    a.k = k; a.importance = importance; a.modality = mod; a.retained = retained; a.evicted = evicted;
+    a.strategy = strategy; a.rn = rn; a.match = match; a.match_sim = match_sim;
+    a.Hkv = p.n_kv_heads; a.D = p.head_dim; a.L = p.seq_len; a.B = p.n_keep; a.E = E;
+    a.tau_eff = tau_effective(p);
+    for (int i = 0; i < 3; ++i) a.ks[i] = p.k_stride[i];
+    const dim3 grid((E + kTile - 1) / kTile, 1, p.n_units * p.n_kv_heads);
+    if (p.dtype == FLOWMM_BF16) match_simt<__nv_bfloat16><<<grid, kSimtThreads, 0, st>>>(a);
+    else match_simt<float><<<grid, kSimtThreads, 0, st>>>(a);
+    FLOWMM_LAUNCH_CHECK();
+    return FLOWMM_OK;
+}
+
+flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, const void *v,
+                        const int32_t *retained, const int32_t *evicted, const int32_t *match, const float *match_sim,
+                        void *k_out, void *v_out, void *ws, cudaStream_t st) {
+    const int E = p.seq_len - p.n_keep, UH = p.n_units * p.n_kv_heads;
+    MergeArgs m;
+    m.k = k; m.v = v; m.k_out = k_out; m.v_out = v_out; m.retained = retained; m.evicted = evicted;
+    m.match_sim = match_sim;
+    m.sorted = nullptr; m.off = nullptr; m.piece_off = nullptr; m.part_off = nullptr;
+    m.partial = at<float>(ws, y.partial);
+    m.Hkv = p.n_kv_heads; m.D = p.head_dim; m.L = p.seq_len; m.B = p.n_keep; m.E = E;
+    m.max_pieces = E == 0 ? p.n_keep : y.max_pieces; m.max_parts = y.max_parts; m.merge_mode = p.merge_mode;
+    for (int i = 0; i < 3; ++i) {
+        m.ks[i] = p.k_stride[i]; m.vs[i] = p.v_stride[i]; m.kos[i] = p.ko_stride[i]; m.vos[i] = p.vo_stride[i];
+    }
+    if (E > 0) {
+        CsrArgs c;
+        c.match = match; c.sort_a = at<int>(ws, y.sort_a); c.sort_b = at<int>(ws, y.sort_b);
+        c.off = at<int>(ws, y.off); c.piece_off = at<int>(ws, y.piece_off); c.part_off = at<int>(ws, y.part_off);
+        c.B = p.n_keep; c.E = E; c.n_pass = y.csr_passes;
+        build_csr_kernel<<<UH, kCsrThreads, 0, st>>>(c);
+        FLOWMM_LAUNCH_CHECK();
+        m.sorted = ((y.csr_passes - 1) & 1) ? c.sort_b : c.sort_a;
+        m.off = c.off; m.piece_off = c.piece_off; m.part_off = c.part_off;
+    }
+    const dim3 gp((m.max_pieces + 7) / 8, UH), gf((p.n_keep + 7) / 8, UH);
+    if (p.dtype == FLOWMM_BF16) {
+        merge_pieces_kernel<__nv_bfloat16><<<gp, 256, 0, st>>>(m);
+        FLOWMM_LAUNCH_CHECK();
+        if (E > kPiece) { merge_finish_kernel<__nv_bfloat16><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCH_CHECK(); }
+    } else {
+        merge_pieces_kernel<float><<<gp, 256, 0, st>>>(m);
+        FLOWMM_LAUNCH_CHECK();
+        if (E > kPiece) { merge_finish_kernel<float><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCH_CHECK(); }
+    }
+    return FLOWMM_OK;
+}
+
+#define FLOWMM_TRY(expr)                         \
+    do {                                         \
+        const flowmm_status _s = (expr);         \
+        if (_s != FLOWMM_OK) return _s;          \
+    } while (0)
+
+}  // namespace
+
+extern "C" {
+
+flowmm_status flowmm_workspace_bytes(const flowmm_params *p, size_t *bytes) {
+    if (!bytes) return FLOWMM_ERR_NULL;
+    FLOWMM_TRY(validate(p));
+    *bytes = make_layout(*p).total;
+    return FLOWMM_OK;
+}
+
+flowmm_status flowmm_score(const flowmm_params *p, const void *q_win, const void *k, const uint8_t *modality,
+                           float *importance, float *cross_mass, void *ws, size_t ws_bytes, void *cuda_stream) {
+    g_launches = 0;
+    FLOWMM_TRY(validate(p));
+    if (!q_win || !k || !modality || !importance || !cross_mass) return FLOWMM_ERR_NULL;
+    if (!aligned16(q_win) || !aligned16(k) || !strides_ok(p->q_stride, p->head_dim) ||
+        !strides_ok(p->k_stride, p->head_dim))
+        return FLOWMM_ERR_ALIGN;
+    Layout y;
+    FLOWMM_TRY(check_ws(p, ws, ws_bytes, y));
+    FLOWMM_TRY(check_device());
+    return run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, static_cast<cudaStream_t>(cuda_stream));
+}
+
+flowmm_status flowmm_layer_flow(const flowmm_params *p, const float *cross_mass, float *rho, int32_t *strategy,
+                                void *cuda_stream) {
+    g_launches = 0;
+    FLOWMM_TRY(validate(p));
+    if (!cross_mass || !rho || !strategy) return FLOWMM_ERR_NULL;
+    FLOWMM_TRY(check_device());
+    return run_layer_flow(*p, cross_mass, rho, strategy, static_cast<cudaStream_t>(cuda_stream));
+}
+
+flowmm_status flowmm_select(const flowmm_params *p, const float *importance, int32_t *retained_idx,
+                            int32_t *evicted_idx, void *ws, size_t ws_bytes, void *cuda_stream) {
+    g_launches = 0;
+    FLOWMM_TRY(validate(p));
+    if (!importance || !retained_idx || (!evicted_idx && p->n_keep < p->seq_len)) return FLOWMM_ERR_NULL;
+    Layout y;
+    FLOWMM_TRY(check_ws(p, ws, ws_bytes, y));
+    FLOWMM_TRY(check_device());
+    return run_select(*p, importance, retained_idx, evicted_idx, static_cast<cudaStream_t>(cuda_stream));
+}
+
+flowmm_status flowmm_match(const flowmm_params *p, const void *k, const float *importance, const uint8_t *modality,
+                           const int32_t *retained_idx, const int32_t *evicted_idx, const int32_t *strategy,
+                           int32_t *match, float *match_sim, void *ws, size_t ws_bytes, void *cuda_stream) {
+    g_launches = 0;
+    FLOWMM_TRY(validate(p));
+    const bool has_e = p->n_keep < p->seq_len;
+    if (!k || !importance || !modality || !retained_idx || !strategy) return FLOWMM_ERR_NULL;
+    if (has_e && (!evicted_idx || !match || !match_sim)) return FLOWMM_ERR_NULL;
+    if (!aligned16(k) || !strides_ok(p->k_stride, p->head_dim)) return FLOWMM_ERR_ALIGN;
+    Layout y;
+    FLOWMM_TRY(check_ws(p, ws, ws_bytes, y));
+    FLOWMM_TRY(check_device());
+    return run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v, const int32_t *retained_idx,
+                           const int32_t *evicted_idx, const int32_t *match, const float *match_sim, void *k_out,
+                           void *v_out, void *ws, size_t ws_bytes, void *cuda_stream) {
+    g_launches = 0;
+    FLOWMM_TRY(validate(p));
+    const bool has_e = p->n_keep < p->seq_len;
+    if (!k || !v || !retained_idx || !k_out || !v_out) return FLOWMM_ERR_NULL;
+    if (has_e && (!evicted_idx || !match || !match_sim)) return FLOWMM_ERR_NULL;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out) ||
+        !strides_ok(p->k_stride, p->head_dim) || !strides_ok(p->v_stride, p->head_dim) ||
+        !strides_ok(p->ko_stride, p->head_dim) || !strides_ok(p->vo_stride, p->head_dim))
+        return FLOWMM_ERR_ALIGN;
+    Layout y;
+    FLOWMM_TRY(check_ws(p, ws, ws_bytes, y));
+    FLOWMM_TRY(check_device());
+    return run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, const void *k, const void *v,
+                                    const uint8_t *modality, void *k_out, void *v_out, float *importance, float *rho,
+                                    int32_t *strategy, int32_t *retained_idx, int32_t *evicted_idx, int32_t *match,
+                                    float *match_sim, void *ws, size_t ws_bytes, void *cuda_stream) {
+    g_launches = 0;
+    FLOWMM_TRY(validate(p));
+    if (!q_win || !k || !v || !modality || !k_out || !v_out) return FLOWMM_ERR_NULL;
+    if (!aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out) ||
+        !strides_ok(p->q_stride, p->head_dim) || !strides_ok(p->k_stride, p->head_dim) ||
+        !strides_ok(p->v_stride, p->head_dim) || !strides_ok(p->ko_stride, p->head_dim) ||
+        !strides_ok(p->vo_stride, p->head_dim))
+        return FLOWMM_ERR_ALIGN;
+    Layout y;
+    FLOWMM_TRY(check_ws(p, ws, ws_bytes, y));
+    FLOWMM_TRY(check_device());
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (!importance) importance = at<float>(ws, y.importance);
+    if (!rho) rho = at<float>(ws, y.rho);
+    if (!strategy) strategy = at<int32_t>(ws, y.strategy);
+    if (!retained_idx) retained_idx = at<int32_t>(ws, y.retained);
+    if (!evicted_idx) evicted_idx = at<int32_t>(ws, y.evicted);
+    if (!match) match = at<int32_t>(ws, y.match);
+    if (!match_sim) match_sim = at<float>(ws, y.match_sim);
+    float *cross_mass = at<float>(ws, y.cross_mass);
+    FLOWMM_TRY(run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, st));
+    FLOWMM_TRY(run_layer_flow(*p, cross_mass, rho, strategy, st));
+    FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st));
+    FLOWMM_TRY(run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws, st));
+    FLOWMM_TRY(run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws, st));
+    return FLOWMM_OK;
+}
+
+flowmm_status flowmm_last_device_status(void *ws, void *cuda_stream) {
+    if (!ws) return FLOWMM_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int32_t word = 0;
+    if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    if (word != 0) {
+        if (cudaMemsetAsync(ws, 0, sizeof(word), st) != cudaSuccess) return FLOWMM_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    }
+    return word >= 0 && word <= FLOWMM_ERR_UNSUPPORTED_DEVICE ? static_cast<flowmm_status>(word) : FLOWMM_ERR_CUDA;
+}
+
+int32_t flowmm_last_launch_count(void) { return g_launches; }
+
+const char *flowmm_status_string(flowmm_status s) {
+    switch (s) {
+        case FLOWMM_OK: return "ok";
+        case FLOWMM_ERR_NULL: return "null pointer";
+        case FLOWMM_ERR_SHAPE: return "inconsistent shape or parameter";
+        case FLOWMM_ERR_BUDGET: return "retention budget out of range";
+        case FLOWMM_ERR_DTYPE: return "unsupported dtype";
+        case FLOWMM_ERR_WORKSPACE: return "workspace too small";
+        case FLOWMM_ERR_ALIGN: return "pointer or stride not aligned";
+        case FLOWMM_ERR_CUDA: return "CUDA error";
+        case FLOWMM_ERR_TIMEOUT: return "device-side wait timed out";
+        case FLOWMM_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.x";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"
