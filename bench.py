@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the FlowMM per-layer KV-cache compression on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--permille 100]
+    python bench.py --impl reference ...       # the fp64 CPU oracle as the reference arm
+
+A step is one flowmm_compress_layer call over every (layer, sequence) unit of
+the workload's stack.  The metric is context tokens compressed per second per
+layer: n_seqs * L * n_layers / step time, summed over GPUs (each GPU compresses
+its own sequences; units are independent, so there is no collective on the
+data path).  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "context tokens compressed/sec per layer (all heads)"
+UNIT = "tokens/s/layer"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--permille", type=int, default=100, help="retention budget in 1/1000 of the context")
+    ap.add_argument("--layers", type=int, default=0, help="use only the first N layers (0 = the whole stack)")
+    ap.add_argument("--path", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-baseline-units", type=int, default=0)
+    return ap.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); smax.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def kernel_model(wl, B, dsize):
+    """Algorithmic flops and bytes of each kernel for ONE unit (all heads), from the
+    operation's definition: what must be read and written once, and the multiply-adds of the
+    two contractions."""
+    Hq, Hkv, L, W, D = wl.n_q_heads, wl.n_kv_heads, wl.seq_len, wl.window, wl.head_dim
+    E = L - B
+    score_flops = 2.0 * Hq * W * L * D
+    score_bytes = (Hkv * L * D + Hq * W * D) * dsize
+    m = {
+        "score_stats": (score_flops, score_bytes),
+        "score_colsum": (score_flops, score_bytes + 4.0 * Hkv * L),
+        "inv_norm": (2.0 * Hkv * L * D, Hkv * L * D * dsize + 4.0 * Hkv * L),
+        "match": (2.0 * Hkv * E * B * D, Hkv * L * D * dsize + 8.0 * Hkv * E),
+        "merge_pieces": (4.0 * Hkv * L * D, 2.0 * Hkv * (L + B) * D * dsize),
+        "select_topb": (0.0, 4.0 * Hkv * L * 2),
+        "build_csr": (0.0, 4.0 * Hkv * E * 3),
+    }
+    return m
+
+
+def model_for(name, model):
+    for key in model:
+        if name.startswith(key):
+            return model[key]
+    return (0.0, 0.0)
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step compresses a bounded sample of the stack."""
+    import numpy as np
+    from oracle import flowmm_oracle as O
+    from paper_2511_05534_b200 import configs, inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = configs.get(args.workload)
+    B = wl.n_keep(args.permille)
+    n_sample = min(wl.n_layers, 8)
+    layers = sorted(set(int(round(i * (wl.n_layers - 1) / max(1, n_sample - 1))) for i in range(n_sample)))
+    if wl.seq_len > 4096:
+        layers = layers[:1]
+    units = [(l, 0) for l in layers]
+    data = inputs.make_units(wl, units)
+    p = O.OracleParams(len(units), wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.seq_len, wl.window, B,
+                       theta=wl.theta, tau=wl.tau_rel, tau_mode=O.TAU_REL)
+    O.build()
+    for _ in range(min(args.warmup, 1)):
+        O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
+    steps = max(1, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
+    dt = (time.perf_counter() - t0) / steps
+    value = wl.seq_len * len(units) / dt
+    sample = "layers %s of the %s stack, one sequence, per step; %d timed steps" % (layers, wl.name, steps)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "budget_permille": args.permille, "n_keep": B, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def cpu_baseline(wl, permille, n_units):
+    import numpy as np
+    from oracle import flowmm_oracle as O
+    from paper_2511_05534_b200 import inputs
+
+    B = wl.n_keep(permille)
+    if n_units <= 0:
+        n_units = wl.n_layers if wl.seq_len <= 1024 else (4 if wl.seq_len <= 4096 else 1)
+    n_units = min(n_units, wl.n_layers)
+    layers = sorted(set(int(round(i * (wl.n_layers - 1) / max(1, n_units - 1))) for i in range(n_units)))
+    units = [(l, 0) for l in layers]
+    data = inputs.make_units(wl, units)
+    p = O.OracleParams(len(units), wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.seq_len, wl.window, B,
+                       theta=wl.theta, tau=wl.tau_rel, tau_mode=O.TAU_REL)
+    O.build()
+    reps, t_total = 0, 0.0
+    while t_total < 10.0 and reps < 20:
+        t0 = time.perf_counter()
+        O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
+        t_total += time.perf_counter() - t0
+        reps += 1
+    dt = t_total / reps
+    return {"value": wl.seq_len * len(units) / dt, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
+            "sample": "%d layer(s) %s of %s, one sequence, %d repetition(s), %.1f s of CPU time" %
+                      (len(units), layers, wl.name, reps, t_total)}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_05534_b200 import binding as F
+    from paper_2511_05534_b200 import build, configs, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    build.build()
+    F.load()
+
+    wl = configs.get(args.workload)
+    n_layers = args.layers if args.layers > 0 else wl.n_layers
+    units = [(l, s) for l in range(n_layers) for s in range(wl.n_seqs)]
+    U = len(units)
+    B = wl.n_keep(args.permille)
+    dt_code = F.BF16 if wl.dtype == "bf16" else F.F32
+    dsize = 2 if wl.dtype == "bf16" else 4
+    p = F.Params(U, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.seq_len, wl.window, B, dtype=dt_code,
+                 theta=wl.theta, tau=wl.tau_rel, tau_mode=F.TAU_REL,
+                 path=F.PATH_SIMT if args.path == "simt" else F.PATH_AUTO)
+
+    # several independent input sets, rotated, so that a step never finds its inputs in L2
+    bytes_per_set = 2 * U * wl.n_kv_heads * wl.seq_len * wl.head_dim * dsize
+    n_sets = max(2, min(8, int(1.5e9 // max(1, bytes_per_set)) + 1))
+    if bytes_per_set > 20e9:
+        n_sets = 1            # a set this large cannot stay in the 126 MB L2 anyway
+    sets = [inputs.make_stack_device(wl, dev, units, seed_offset=rank * 100 + i) for i in range(n_sets)]
+    k_out = torch.empty((U, wl.n_kv_heads, B, wl.head_dim), dtype=sets[0][1].dtype, device=dev)
+    v_out = torch.empty_like(k_out)
+    ws = F.alloc_workspace(p, dev)
+
+    def step(i):
+        q, k, v, m = sets[i % n_sets]
+        F.flowmm_compress_layer(p, q, k, v, m, k_out, v_out, ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    launches_per_step = F.flowmm_last_launch_count()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    status = F.flowmm_last_device_status(ws)
+    if status != 0:
+        raise RuntimeError("device status: " + F.status_string(status))
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    tokens_layers = wl.n_seqs * wl.seq_len * n_layers        # tokens x layers compressed per step per GPU
+    value = world * tokens_layers / (ms_step * 1e-3)
+
+    # per-kernel attribution: the same steps again with an event after every kernel
+    F.flowmm_profile_enable(True)
+    per_kernel = {}
+    for i in range(args.steps):
+        step(i)
+        for name, ms in F.flowmm_profile_read():
+            per_kernel.setdefault(name, []).append(ms)
+    F.flowmm_profile_enable(False)
+    torch.cuda.synchronize()
+    peaks = load_peaks()
+    model = kernel_model(wl, B, dsize)
+    kernels = {}
+    for name, times in per_kernel.items():
+        avg = sum(times) / len(times)
+        flops, nbytes = model_for(name, model)
+        flops, nbytes = flops * U, nbytes * U
+        t_tensor = flops / (peaks["bf16_tflops_sustained"] * 1e12) if dt_code == F.BF16 else 0.0
+        t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+        bound = "tensor" if t_tensor > t_hbm else "hbm"
+        kernels[name] = {"ms": avg, "bound": bound, "gbs": nbytes / (avg * 1e-3) / 1e9,
+                         "tflops": flops / (avg * 1e-3) / 1e12,
+                         "frac": (t_tensor if bound == "tensor" else t_hbm) / (avg * 1e-3)}
+    top = max(kernels, key=lambda n: kernels[n]["ms"])
+    tk = kernels[top]
+    if tk["bound"] == "tensor":
+        roofline = {"kernel": top, "bound": "tensor", "achieved": tk["tflops"], "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": tk["frac"], "traffic": None,
+                    "peak_source": peaks["source"] + " (sustained bf16)"}
+    else:
+        roofline = {"kernel": top, "bound": "hbm", "achieved": tk["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": tk["frac"], "traffic": None, "peak_source": peaks["source"]}
+    roofline["launch_ms"] = tk["ms"]
+
+    # end to end: pinned host inputs -> device -> compress -> pinned host result, every step
+    hq, hk, hv, hm = (t.cpu().pin_memory() for t in sets[0])
+    dq, dk, dv, dm = (torch.empty_like(t) for t in sets[0])
+    hko, hvo = torch.empty_like(k_out, device="cpu").pin_memory(), torch.empty_like(v_out, device="cpu").pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hm))
+    d2h = sum(t.numel() * t.element_size() for t in (hko, hvo))
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True)
+        dv.copy_(hv, non_blocking=True); dm.copy_(hm, non_blocking=True)
+        F.flowmm_compress_layer(p, dq, dk, dv, dm, k_out, v_out, ws)
+        hko.copy_(k_out, non_blocking=True); hvo.copy_(v_out, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * tokens_layers / (e2e_ms / e2e_steps * 1e-3)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "layers": n_layers, "seqs": wl.n_seqs, "n_q_heads": wl.n_q_heads,
+                       "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "seq_len": wl.seq_len,
+                       "window": wl.window, "budget_permille": args.permille, "n_keep": B,
+                       "units_per_call": U, "l2": "%d rotating input sets of %.0f MB (inputs larger than L2)" %
+                       (n_sets, bytes_per_set / 1e6), "path": args.path, "parallelism": "units sharded, no collective"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline,
+            "kernels": {n: {k2: (round(v2, 5) if isinstance(v2, float) else v2) for k2, v2 in d.items()}
+                        for n, d in kernels.items()},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl, args.permille, args.cpu_baseline_units)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -170,6 +170,17 @@ flowmm_status flowmm_last_device_status(void *ws, void *cuda_stream);
 /* Number of kernels the most recent compute entry point of this thread enqueued. */
 int32_t flowmm_last_launch_count(void);
 
+/*
+ * Profiling aid, per host thread, off by default.  While on, every compute entry point records
+ * a CUDA event on its stream before its first kernel and after each kernel (one extra event
+ * record per launch).  flowmm_profile_read waits for the last of them and fills, in launch
+ * order, a static kernel name and the kernel's duration in milliseconds for the most recent
+ * entry point; it returns the number of entries written (0 when off, -1 on a CUDA error).
+ * The first enable creates the events.
+ */
+flowmm_status flowmm_profile_enable(int32_t on);
+int32_t flowmm_profile_read(const char **names, float *ms, int32_t max_entries);
+
 /* Static, human-readable name of a status code. */
 const char *flowmm_status_string(flowmm_status s);
 

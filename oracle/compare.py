@@ -62,9 +62,12 @@ def check_structure(p: O.OracleParams, g: Dict[str, np.ndarray], modality: np.nd
     _require(np.all(np.diff(ret, axis=-1) > 0) and (L - B < 2 or np.all(np.diff(evi, axis=-1) > 0)),
              "index lists must ascend")
     if L > B:
-        lo = np.take_along_axis(imp, ret.astype(np.int64), -1).min(-1)
+        piv_imp = np.take_along_axis(imp, ret.astype(np.int64), -1)
+        if p.keep_window:                      # forced window pivots are exempt from the ranking
+            piv_imp = np.where(ret >= L - W, np.inf, piv_imp)
+            _require(np.all((ret >= L - W).sum(-1) == W), "keep_window: a proxy token was evicted")
         hi = np.take_along_axis(imp, evi.astype(np.int64), -1).max(-1)
-        _require(np.all(lo >= hi), "a non-pivot outranks a pivot")
+        _require(np.all(piv_imp.min(-1) >= hi), "a non-pivot outranks a pivot")
         mt = g["match"]
         _require(np.all((mt >= -1) & (mt < B)), "match out of range")
         _require(np.all(np.abs(g["match_sim"]) <= 1 + 1e-5), "cosine outside [-1, 1]")
@@ -106,7 +109,11 @@ def compare(p: O.OracleParams, q, k, v, modality, g: Dict[str, np.ndarray], bf16
             if np.array_equal(ret[u, h], g["retained"][u, h]):
                 continue
             diff = np.setxor1d(ret[u, h], g["retained"][u, h])
-            bound = np.sort(imp[u, h])[::-1][B - 1]
+            if p.keep_window:                  # the boundary among the tokens that compete for a place
+                free = imp[u, h][: L - p.window]
+                bound = np.sort(free)[::-1][B - p.window - 1] if B > p.window else np.inf
+            else:
+                bound = np.sort(imp[u, h])[::-1][B - 1]
             _require(np.all(np.abs(imp[u, h][diff] - bound) <= GAP_RTOL * bound),
                      "pivot set differs away from the top-B boundary (unit %d head %d)" % (u, h))
             n_set_ties += len(diff) // 2

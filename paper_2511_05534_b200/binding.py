@@ -28,6 +28,7 @@ PATH_AUTO, PATH_SIMT = 0, 1
 EXPORTS = (
     "flowmm_workspace_bytes", "flowmm_score", "flowmm_layer_flow", "flowmm_select", "flowmm_match", "flowmm_merge",
     "flowmm_compress_layer", "flowmm_last_device_status", "flowmm_last_launch_count", "flowmm_status_string",
+    "flowmm_profile_enable", "flowmm_profile_read",
 )
 
 
@@ -113,6 +114,8 @@ def load() -> ctypes.CDLL:
             getattr(lib, name)
         lib.flowmm_status_string.restype = ctypes.c_char_p
         lib.flowmm_last_launch_count.restype = ctypes.c_int32
+        lib.flowmm_profile_enable.restype = ctypes.c_int
+        lib.flowmm_profile_read.restype = ctypes.c_int32
         for name in EXPORTS[:8]:
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
@@ -205,6 +208,20 @@ def flowmm_last_device_status(ws) -> int:
 
 def flowmm_last_launch_count() -> int:
     return int(load().flowmm_last_launch_count())
+
+
+def flowmm_profile_enable(on: bool):
+    _check(load().flowmm_profile_enable(ctypes.c_int32(1 if on else 0)), "flowmm_profile_enable")
+
+
+def flowmm_profile_read(max_entries: int = 32):
+    """[(kernel name, milliseconds), ...] of the most recent entry point, in launch order."""
+    names = (ctypes.c_char_p * max_entries)()
+    ms = (ctypes.c_float * max_entries)()
+    n = load().flowmm_profile_read(names, ms, ctypes.c_int32(max_entries))
+    if n < 0:
+        raise FlowmmError(7, "flowmm_profile_read")
+    return [(names[i].decode(), float(ms[i])) for i in range(n)]
 
 
 def compress_layer_alloc(p: Params, q_win, k, v, modality, ws=None, diagnostics=True):

@@ -16,10 +16,33 @@ namespace {
 
 thread_local int32_t g_launches = 0;
 
-#define FLOWMM_LAUNCH_CHECK()                                   \
-    do {                                                        \
-        ++g_launches;                                           \
+// Optional per-kernel timing: one event before the first kernel of an entry point, one after each.
+constexpr int kMaxProfiled = 32;
+struct Profile {
+    bool on = false, have_events = false;
+    cudaEvent_t ev[kMaxProfiled + 1];
+    const char *name[kMaxProfiled];
+    int n = 0;
+};
+thread_local Profile g_prof;
+
+inline void profile_begin(cudaStream_t st) {
+    g_launches = 0;
+    g_prof.n = 0;
+    if (g_prof.on) cudaEventRecord(g_prof.ev[0], st);
+}
+inline void profile_mark(const char *name, cudaStream_t st) {
+    if (g_prof.on && g_prof.n < kMaxProfiled) {
+        g_prof.name[g_prof.n] = name;
+        cudaEventRecord(g_prof.ev[++g_prof.n], st);
+    }
+}
+
+#define FLOWMM_LAUNCHED(name)                                          \
+    do {                                                               \
+        ++g_launches;                                                  \
         if (cudaGetLastError() != cudaSuccess) return FLOWMM_ERR_CUDA; \
+        profile_mark(name, st);                                        \
     } while (0)
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -142,18 +165,18 @@ flowmm_status run_score(const flowmm_params &p, const Layout &y, const void *q, 
     const size_t dyn = (size_t)3 * GW * sizeof(float);
     if (p.dtype == FLOWMM_BF16) {
         score_stats_simt<__nv_bfloat16><<<g1, kSimtThreads, 0, st>>>(a);
-        FLOWMM_LAUNCH_CHECK();
+        FLOWMM_LAUNCHED("score_stats_simt");
         score_colsum_simt<__nv_bfloat16><<<g2, kSimtThreads, dyn, st>>>(a);
-        FLOWMM_LAUNCH_CHECK();
+        FLOWMM_LAUNCHED("score_colsum_simt");
     } else {
         score_stats_simt<float><<<g1, kSimtThreads, 0, st>>>(a);
-        FLOWMM_LAUNCH_CHECK();
+        FLOWMM_LAUNCHED("score_stats_simt");
         score_colsum_simt<float><<<g2, kSimtThreads, dyn, st>>>(a);
-        FLOWMM_LAUNCH_CHECK();
+        FLOWMM_LAUNCHED("score_colsum_simt");
     }
     const int n = p.n_units * p.n_q_heads;
     cross_mass_reduce<<<(n + 255) / 256, 256, 0, st>>>(a.cross_part, y.n_chunk2, n, cross_mass);
-    FLOWMM_LAUNCH_CHECK();
+    FLOWMM_LAUNCHED("cross_mass_reduce");
     return FLOWMM_OK;
 }
 
@@ -161,7 +184,7 @@ flowmm_status run_layer_flow(const flowmm_params &p, const float *cross_mass, fl
                              cudaStream_t st) {
     layer_flow_kernel<<<(p.n_units + 127) / 128, 128, 0, st>>>(cross_mass, p.n_units, p.n_q_heads, p.window, p.theta,
                                                                 p.flow_mode, rho, strategy);
-    FLOWMM_LAUNCH_CHECK();
+    FLOWMM_LAUNCHED("layer_flow");
     return FLOWMM_OK;
 }
 
@@ -169,7 +192,7 @@ flowmm_status run_select(const flowmm_params &p, const float *importance, int32_
                          cudaStream_t st) {
     select_topb_kernel<<<p.n_units * p.n_kv_heads, kSelectThreads, 0, st>>>(importance, p.seq_len, p.n_keep, p.window,
                                                                            p.keep_window, retained, evicted);
-    FLOWMM_LAUNCH_CHECK();
+    FLOWMM_LAUNCHED("select_topb");
     return FLOWMM_OK;
 }
 
@@ -189,7 +212,7 @@ flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, 
     else
         inv_norm_kernel<float><<<blocks, 256, 0, st>>>(k, rows, p.n_kv_heads, p.seq_len, p.head_dim, p.k_stride[0],
                                                        p.k_stride[1], p.k_stride[2], rn);
-    FLOWMM_LAUNCH_CHECK();
+    FLOWMM_LAUNCHED("inv_norm");
     MatchArgs a;
     a.k = k; a.importance = importance; a.modality = mod; a.retained = retained; a.evicted = evicted;
     a.strategy = strategy; a.rn = rn; a.match = match; a.match_sim = match_sim;
@@ -199,7 +222,7 @@ flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, 
     const dim3 grid((E + kTile - 1) / kTile, 1, p.n_units * p.n_kv_heads);
     if (p.dtype == FLOWMM_BF16) match_simt<__nv_bfloat16><<<grid, kSimtThreads, 0, st>>>(a);
     else match_simt<float><<<grid, kSimtThreads, 0, st>>>(a);
-    FLOWMM_LAUNCH_CHECK();
+    FLOWMM_LAUNCHED("match_simt");
     return FLOWMM_OK;
 }
 
@@ -223,19 +246,19 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
         c.off = at<int>(ws, y.off); c.piece_off = at<int>(ws, y.piece_off); c.part_off = at<int>(ws, y.part_off);
         c.B = p.n_keep; c.E = E; c.n_pass = y.csr_passes;
         build_csr_kernel<<<UH, kCsrThreads, 0, st>>>(c);
-        FLOWMM_LAUNCH_CHECK();
+        FLOWMM_LAUNCHED("build_csr");
         m.sorted = ((y.csr_passes - 1) & 1) ? c.sort_b : c.sort_a;
         m.off = c.off; m.piece_off = c.piece_off; m.part_off = c.part_off;
     }
     const dim3 gp((m.max_pieces + 7) / 8, UH), gf((p.n_keep + 7) / 8, UH);
     if (p.dtype == FLOWMM_BF16) {
         merge_pieces_kernel<__nv_bfloat16><<<gp, 256, 0, st>>>(m);
-        FLOWMM_LAUNCH_CHECK();
-        if (E > kPiece) { merge_finish_kernel<__nv_bfloat16><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCH_CHECK(); }
+        FLOWMM_LAUNCHED("merge_pieces");
+        if (E > kPiece) { merge_finish_kernel<__nv_bfloat16><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCHED("merge_finish"); }
     } else {
         merge_pieces_kernel<float><<<gp, 256, 0, st>>>(m);
-        FLOWMM_LAUNCH_CHECK();
-        if (E > kPiece) { merge_finish_kernel<float><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCH_CHECK(); }
+        FLOWMM_LAUNCHED("merge_pieces");
+        if (E > kPiece) { merge_finish_kernel<float><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCHED("merge_finish"); }
     }
     return FLOWMM_OK;
 }
@@ -259,7 +282,7 @@ flowmm_status flowmm_workspace_bytes(const flowmm_params *p, size_t *bytes) {
 
 flowmm_status flowmm_score(const flowmm_params *p, const void *q_win, const void *k, const uint8_t *modality,
                            float *importance, float *cross_mass, void *ws, size_t ws_bytes, void *cuda_stream) {
-    g_launches = 0;
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
     FLOWMM_TRY(validate(p));
     if (!q_win || !k || !modality || !importance || !cross_mass) return FLOWMM_ERR_NULL;
     if (!aligned16(q_win) || !aligned16(k) || !strides_ok(p->q_stride, p->head_dim) ||
@@ -273,7 +296,7 @@ flowmm_status flowmm_score(const flowmm_params *p, const void *q_win, const void
 
 flowmm_status flowmm_layer_flow(const flowmm_params *p, const float *cross_mass, float *rho, int32_t *strategy,
                                 void *cuda_stream) {
-    g_launches = 0;
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
     FLOWMM_TRY(validate(p));
     if (!cross_mass || !rho || !strategy) return FLOWMM_ERR_NULL;
     FLOWMM_TRY(check_device());
@@ -282,7 +305,7 @@ flowmm_status flowmm_layer_flow(const flowmm_params *p, const float *cross_mass,
 
 flowmm_status flowmm_select(const flowmm_params *p, const float *importance, int32_t *retained_idx,
                             int32_t *evicted_idx, void *ws, size_t ws_bytes, void *cuda_stream) {
-    g_launches = 0;
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
     FLOWMM_TRY(validate(p));
     if (!importance || !retained_idx || (!evicted_idx && p->n_keep < p->seq_len)) return FLOWMM_ERR_NULL;
     Layout y;
@@ -294,7 +317,7 @@ flowmm_status flowmm_select(const flowmm_params *p, const float *importance, int
 flowmm_status flowmm_match(const flowmm_params *p, const void *k, const float *importance, const uint8_t *modality,
                            const int32_t *retained_idx, const int32_t *evicted_idx, const int32_t *strategy,
                            int32_t *match, float *match_sim, void *ws, size_t ws_bytes, void *cuda_stream) {
-    g_launches = 0;
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
     FLOWMM_TRY(validate(p));
     const bool has_e = p->n_keep < p->seq_len;
     if (!k || !importance || !modality || !retained_idx || !strategy) return FLOWMM_ERR_NULL;
@@ -310,7 +333,7 @@ flowmm_status flowmm_match(const flowmm_params *p, const void *k, const float *i
 flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v, const int32_t *retained_idx,
                            const int32_t *evicted_idx, const int32_t *match, const float *match_sim, void *k_out,
                            void *v_out, void *ws, size_t ws_bytes, void *cuda_stream) {
-    g_launches = 0;
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
     FLOWMM_TRY(validate(p));
     const bool has_e = p->n_keep < p->seq_len;
     if (!k || !v || !retained_idx || !k_out || !v_out) return FLOWMM_ERR_NULL;
@@ -330,7 +353,7 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
                                     const uint8_t *modality, void *k_out, void *v_out, float *importance, float *rho,
                                     int32_t *strategy, int32_t *retained_idx, int32_t *evicted_idx, int32_t *match,
                                     float *match_sim, void *ws, size_t ws_bytes, void *cuda_stream) {
-    g_launches = 0;
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
     FLOWMM_TRY(validate(p));
     if (!q_win || !k || !v || !modality || !k_out || !v_out) return FLOWMM_ERR_NULL;
     if (!aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out) ||
@@ -372,6 +395,28 @@ flowmm_status flowmm_last_device_status(void *ws, void *cuda_stream) {
 }
 
 int32_t flowmm_last_launch_count(void) { return g_launches; }
+
+flowmm_status flowmm_profile_enable(int32_t on) {
+    if (on && !g_prof.have_events) {
+        for (int i = 0; i <= kMaxProfiled; ++i)
+            if (cudaEventCreate(&g_prof.ev[i]) != cudaSuccess) return FLOWMM_ERR_CUDA;
+        g_prof.have_events = true;
+    }
+    g_prof.on = on != 0;
+    g_prof.n = 0;
+    return FLOWMM_OK;
+}
+
+int32_t flowmm_profile_read(const char **names, float *ms, int32_t max_entries) {
+    if (!g_prof.on || g_prof.n == 0) return 0;
+    if (cudaEventSynchronize(g_prof.ev[g_prof.n]) != cudaSuccess) return -1;
+    const int n = g_prof.n < max_entries ? g_prof.n : max_entries;
+    for (int i = 0; i < n; ++i) {
+        if (names) names[i] = g_prof.name[i];
+        if (ms && cudaEventElapsedTime(&ms[i], g_prof.ev[i], g_prof.ev[i + 1]) != cudaSuccess) return -1;
+    }
+    return n;
+}
 
 const char *flowmm_status_string(flowmm_status s) {
     switch (s) {
