@@ -31,11 +31,12 @@ UNIT = "tokens/s/layer"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--permille", type=int, default=100, help="retention budget in 1/1000 of the context")
+    ap.add_argument("--permille", type=int, default=0,
+                    help="retention budget in 1/1000 of the context (0: 100 if the workload lists it, else its first)")
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers (0 = the whole stack)")
     ap.add_argument("--path", default="auto", choices=["auto", "simt"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -53,47 +54,56 @@ def load_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """SM clock and throttle-reason samples taken through NVML while the timed region runs
+    (read-only queries, a few milliseconds apart, from a helper thread)."""
 
     def __init__(self, gpu_index: int):
-        self.proc = None
         self.gpu = gpu_index
+        self.samples, self.reasons = [], set()
+        self.sm_max = None
+        self._stop = False
+        self._thread = None
+        self._err = None
+
+    def _run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.gpu
+            if vis:
+                ids = [x for x in vis.split(",") if x.strip() != ""]
+                if self.gpu < len(ids) and ids[self.gpu].strip().isdigit():
+                    idx = int(ids[self.gpu])
+            h = nv.nvmlDeviceGetHandleByIndex(idx)
+            self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+            get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            table = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+            while not self._stop:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                bits = int(get_reasons(h))
+                for bit, name in table.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+                time.sleep(0.002)
+        except Exception as exc:            # NVML missing or refused: report it, do not fail the run
+            self._err = repr(exc)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+        import threading
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
-            parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 9:
-                continue
-            try:
-                sm.append(float(parts[1])); smax.append(float(parts[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop = True
+        if self._thread is not None:
+            self._thread.join(timeout=5)
+        out = {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.sm_max,
+               "samples": len(self.samples), "reasons": sorted(self.reasons)}
+        if self._err:
+            out["error"] = self._err
+        return out
 
 
 def kernel_model(wl, B, dsize):
@@ -116,11 +126,16 @@ def kernel_model(wl, B, dsize):
     return m
 
 
+KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
+    "score_stats_simt": "score_stats", "score_stats_tc": "score_stats",
+    "score_colsum_simt": "score_colsum", "score_colsum_tc": "score_colsum",
+    "inv_norm": "inv_norm", "match_simt": "match", "match_tc": "match", "merge_pieces": "merge_pieces",
+    "select_topb": "select_topb", "build_csr": "build_csr",
+}
+
+
 def model_for(name, model):
-    for key in model:
-        if name.startswith(key):
-            return model[key]
-    return (0.0, 0.0)
+    return model.get(KERNEL_MODEL.get(name, ""), (0.0, 0.0))
 
 
 def run_reference(args):
@@ -134,7 +149,7 @@ def run_reference(args):
         return
     wl = configs.get(args.workload)
     B = wl.n_keep(args.permille)
-    n_sample = min(wl.n_layers, 8)
+    n_sample = min(wl.n_layers, 8 if wl.seq_len <= 1024 else 2)
     layers = sorted(set(int(round(i * (wl.n_layers - 1) / max(1, n_sample - 1))) for i in range(n_sample)))
     if wl.seq_len > 4096:
         layers = layers[:1]
@@ -143,9 +158,9 @@ def run_reference(args):
     p = O.OracleParams(len(units), wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.seq_len, wl.window, B,
                        theta=wl.theta, tau=wl.tau_rel, tau_mode=O.TAU_REL)
     O.build()
-    for _ in range(min(args.warmup, 1)):
+    for _ in range(args.warmup):
         O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
-    steps = max(1, min(args.steps, 10))
+    steps = max(1, args.steps)
     t0 = time.perf_counter()
     for _ in range(steps):
         O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
@@ -154,7 +169,7 @@ def run_reference(args):
     sample = "layers %s of the %s stack, one sequence, per step; %d timed steps" % (layers, wl.name, steps)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "budget_permille": args.permille, "n_keep": B, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.threads(), "kind": "oracle", "sample": sample},
@@ -352,6 +367,10 @@ def run_ours(args):
 
 def main():
     args = parse_args()
+    if args.permille <= 0:
+        from paper_2511_05534_b200 import configs
+        budgets = configs.get(args.workload).budgets_permille
+        args.permille = 100 if 100 in budgets else budgets[0]
     if args.impl == "reference":
         run_reference(args)
     else:

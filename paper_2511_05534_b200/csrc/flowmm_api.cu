@@ -7,8 +7,10 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "match_tc.cuh"
 #include "select_merge.cuh"
 #include "simt_kernels.cuh"
+#include "tc_host.cuh"
 
 using namespace flowmm;
 
@@ -51,8 +53,9 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
     size_t row_part, cross_part, rn, sort_a, sort_b, off, piece_off, part_off, partial;
+    size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod;
     size_t total;
-    int n_chunk1, chunk1, n_chunk2, chunk2, max_pieces, max_parts, csr_passes;
+    int n_chunk1, chunk1, n_chunk2, chunk2, max_pieces, max_parts, csr_passes, c_tot, n_rt;
 };
 
 int chunks_for(int L, int other_ctas, int &chunk) {
@@ -96,6 +99,14 @@ Layout make_layout(const flowmm_params &p) {
     y.piece_off = take(U * Hkv * (B + 1) * 4);
     y.part_off = take(U * Hkv * (B + 1) * 4);
     y.partial = take(U * Hkv * (size_t)y.max_parts * (2 * D + 4) * 4);
+    y.c_tot = (int)((B + 31) / 32 * 32 + 32);
+    y.n_rt = (int)((L + kMtRows - 1) / kMtRows);
+    y.cand_k = take(U * Hkv * (size_t)y.c_tot * 128 * 2);
+    y.cand_scale = take(U * Hkv * (size_t)y.c_tot * 4);
+    y.cand_slot = take(U * Hkv * (size_t)y.c_tot * 4);
+    y.cand_count = take(U * Hkv * 2 * 4);
+    y.rank = take(U * Hkv * L * 4);
+    y.tile_mod = take(U * (size_t)y.n_rt);
     y.total = o;
     return y;
 }
@@ -196,6 +207,47 @@ flowmm_status run_select(const flowmm_params &p, const float *importance, int32_
     return FLOWMM_OK;
 }
 
+bool use_tc(const flowmm_params &p) {
+    return p.path == FLOWMM_PATH_AUTO && p.dtype == FLOWMM_BF16 && p.head_dim == 128;
+}
+
+flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
+                           const uint8_t *mod, const int32_t *retained, const int32_t *evicted,
+                           const int32_t *strategy, int32_t *match, float *match_sim, void *ws, cudaStream_t st) {
+    const int UH = p.n_units * p.n_kv_heads, E = p.seq_len - p.n_keep;
+    MatchPrepArgs g;
+    g.k = k; g.importance = importance; g.rn = at<float>(ws, y.rn); g.modality = mod;
+    g.retained = retained; g.evicted = evicted;
+    g.cand_k = at<__nv_bfloat16>(ws, y.cand_k); g.cand_scale = at<float>(ws, y.cand_scale);
+    g.cand_slot = at<int>(ws, y.cand_slot); g.cand_count = at<int>(ws, y.cand_count);
+    g.rank = at<int>(ws, y.rank); g.tile_mod = at<uint8_t>(ws, y.tile_mod);
+    g.Hkv = p.n_kv_heads; g.L = p.seq_len; g.B = p.n_keep; g.E = E; g.Ctot = y.c_tot; g.n_rt = y.n_rt;
+    g.tau_eff = tau_effective(p);
+    for (int i = 0; i < 3; ++i) g.ks[i] = p.k_stride[i];
+    match_prepare_kernel<<<UH, 256, 0, st>>>(g);
+    FLOWMM_LAUNCHED("match_prepare");
+
+    CUtensorMap k_map, cand_map;
+    const uint64_t kd[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
+    const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
+    const uint64_t cd[3] = {128, (uint64_t)y.c_tot, (uint64_t)UH};
+    const uint64_t cs[2] = {256, (uint64_t)y.c_tot * 256};
+    if (!tc::make_bf16_map(&k_map, k, 4, kd, ks, kMtRows) || !tc::make_bf16_map(&cand_map, g.cand_k, 3, cd, cs, kMtCols))
+        return FLOWMM_ERR_CUDA;
+    MatchTcArgs a;
+    a.cand_count = g.cand_count; a.cand_slot = g.cand_slot; a.rank = g.rank; a.strategy = strategy;
+    a.cand_scale = g.cand_scale; a.rn = g.rn; a.modality = mod; a.tile_mod = g.tile_mod;
+    a.match = match; a.match_sim = match_sim; a.status = at<int>(ws, y.status);
+    a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.E = E; a.Ctot = y.c_tot; a.n_rt = y.n_rt; a.n_items = UH * y.n_rt;
+    if (cudaFuncSetAttribute(match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMtSmemBytes) !=
+        cudaSuccess)
+        return FLOWMM_ERR_CUDA;
+    const int grid = a.n_items < tc::sm_count() ? a.n_items : tc::sm_count();
+    match_tc_kernel<<<grid, kMtThreads, kMtSmemBytes, st>>>(k_map, cand_map, a);
+    FLOWMM_LAUNCHED("match_tc");
+    return FLOWMM_OK;
+}
+
 flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
                         const uint8_t *mod, const int32_t *retained, const int32_t *evicted, const int32_t *strategy,
                         int32_t *match, float *match_sim, void *ws, cudaStream_t st) {
@@ -213,6 +265,7 @@ flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, 
         inv_norm_kernel<float><<<blocks, 256, 0, st>>>(k, rows, p.n_kv_heads, p.seq_len, p.head_dim, p.k_stride[0],
                                                        p.k_stride[1], p.k_stride[2], rn);
     FLOWMM_LAUNCHED("inv_norm");
+    if (use_tc(p)) return run_match_tc(p, y, k, importance, mod, retained, evicted, strategy, match, match_sim, ws, st);
     MatchArgs a;
     a.k = k; a.importance = importance; a.modality = mod; a.retained = retained; a.evicted = evicted;
     a.strategy = strategy; a.rn = rn; a.match = match; a.match_sim = match_sim;
