@@ -8,6 +8,7 @@
 
 #include "common.cuh"
 #include "match_tc.cuh"
+#include "score_tc.cuh"
 #include "select_merge.cuh"
 #include "simt_kernels.cuh"
 #include "tc_host.cuh"
@@ -53,7 +54,8 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
     size_t row_part, cross_part, rn, sort_a, sort_b, off, piece_off, part_off, partial;
-    size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod;
+    size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod, negc;
+    int tc_n_qt, tc_n_chunk, tc_tiles_per_chunk, gw_pad;
     size_t total;
     int n_chunk1, chunk1, n_chunk2, chunk2, max_pieces, max_parts, csr_passes, c_tot, n_rt;
 };
@@ -90,8 +92,21 @@ Layout make_layout(const flowmm_params &p) {
     y.evicted = take(U * Hkv * E * 4);
     y.match = take(U * Hkv * E * 4);
     y.match_sim = take(U * Hkv * E * 4);
-    y.row_part = take(U * Hq * W * (size_t)y.n_chunk1 * 8);
-    y.cross_part = take(U * Hq * (size_t)y.n_chunk2 * 4);
+    y.n_rt = (int)((L + tcs::kRows - 1) / tcs::kRows);
+    {   // pass 1 of the tensor-core scoring: key chunks of whole 256-key tiles
+        y.tc_n_qt = (int)((G * W + tcs::kRows - 1) / tcs::kRows);
+        const int key_tiles = (int)((L + tcs::kCols - 1) / tcs::kCols);
+        int want = (int)((2 * 148 + U * Hkv * y.tc_n_qt - 1) / (U * Hkv * y.tc_n_qt));
+        want = want < 1 ? 1 : (want > key_tiles ? key_tiles : want);
+        y.tc_tiles_per_chunk = (key_tiles + want - 1) / want;
+        y.tc_n_chunk = (key_tiles + y.tc_tiles_per_chunk - 1) / y.tc_tiles_per_chunk;
+        y.gw_pad = (int)((G * W + tcs::kCols - 1) / tcs::kCols * tcs::kCols);
+    }
+    const size_t max_chunk1 = (size_t)(y.n_chunk1 > y.tc_n_chunk ? y.n_chunk1 : y.tc_n_chunk);
+    const size_t max_chunk2 = (size_t)(y.n_chunk2 > 4 * y.n_rt ? y.n_chunk2 : 4 * y.n_rt);
+    y.row_part = take(U * Hq * W * max_chunk1 * 8);
+    y.cross_part = take(U * Hq * max_chunk2 * 4);
+    y.negc = take(U * Hkv * (size_t)y.gw_pad * 4);
     y.rn = take(U * Hkv * L * 4);
     y.sort_a = take(U * Hkv * E * 4);
     y.sort_b = take(U * Hkv * E * 4);
@@ -100,7 +115,6 @@ Layout make_layout(const flowmm_params &p) {
     y.part_off = take(U * Hkv * (B + 1) * 4);
     y.partial = take(U * Hkv * (size_t)y.max_parts * (2 * D + 4) * 4);
     y.c_tot = (int)((B + 31) / 32 * 32 + 32);
-    y.n_rt = (int)((L + kMtRows - 1) / kMtRows);
     y.cand_k = take(U * Hkv * (size_t)y.c_tot * 128 * 2);
     y.cand_scale = take(U * Hkv * (size_t)y.c_tot * 4);
     y.cand_slot = take(U * Hkv * (size_t)y.c_tot * 4);
@@ -158,8 +172,60 @@ float tau_effective(const flowmm_params &p) {
 
 // ---- step launchers (no validation; the entry points below validate) --------------------------
 
+bool use_tc(const flowmm_params &p) {
+    return p.path == FLOWMM_PATH_AUTO && p.dtype == FLOWMM_BF16 && p.head_dim == 128;
+}
+bool use_tc_score(const flowmm_params &p) {
+    const int gw = p.n_q_heads / p.n_kv_heads * p.window;
+    return use_tc(p) && (p.window == 32 || p.window == 64 || p.window == 128) && gw <= 1024;
+}
+
+flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
+                           float *importance, float *cross_mass, void *ws, cudaStream_t st) {
+    const int UH = p.n_units * p.n_kv_heads, G = p.n_q_heads / p.n_kv_heads, W = p.window;
+    ScoreTcArgs a;
+    a.row_part = at<float2>(ws, y.row_part); a.negc = at<float>(ws, y.negc); a.modality = mod;
+    a.importance = importance; a.cross_part = at<float>(ws, y.cross_part); a.status = at<int>(ws, y.status);
+    a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.G = G; a.W = W; a.L = p.seq_len; a.GW = G * W; a.GWpad = y.gw_pad;
+    a.n_qt = y.tc_n_qt; a.n_chunk = y.tc_n_chunk; a.tiles_per_chunk = y.tc_tiles_per_chunk; a.n_rt = y.n_rt;
+    a.a_heads = G < tcs::kRows / W ? G : tcs::kRows / W;
+    a.b_heads = G < tcs::kCols / W ? G : tcs::kCols / W;
+    a.n_items1 = UH * a.n_qt * a.n_chunk; a.n_items2 = UH * a.n_rt;
+    const float scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * kLog2e;
+
+    CUtensorMap qa, qb, k128, k256;
+    const uint64_t qd[4] = {128, (uint64_t)W, (uint64_t)p.n_q_heads, (uint64_t)p.n_units};
+    const uint64_t qs[3] = {(uint64_t)p.q_stride[2] * 2, (uint64_t)p.q_stride[1] * 2, (uint64_t)p.q_stride[0] * 2};
+    const uint64_t kd[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
+    const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
+    const uint32_t bqa[4] = {64, (uint32_t)W, (uint32_t)a.a_heads, 1}, bqb[4] = {64, (uint32_t)W, (uint32_t)a.b_heads, 1};
+    const uint32_t bk128[4] = {64, tcs::kRows, 1, 1}, bk256[4] = {64, tcs::kCols, 1, 1};
+    if (!tc::make_bf16_map(&qa, q, 4, qd, qs, bqa) || !tc::make_bf16_map(&qb, q, 4, qd, qs, bqb) ||
+        !tc::make_bf16_map(&k128, k, 4, kd, ks, bk128) || !tc::make_bf16_map(&k256, k, 4, kd, ks, bk256))
+        return FLOWMM_ERR_CUDA;
+    if (cudaFuncSetAttribute(score_stats_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(score_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::kSmemBytes) != cudaSuccess)
+        return FLOWMM_ERR_CUDA;
+    const int sms = tc::sm_count();
+    score_stats_tc_kernel<<<a.n_items1 < sms ? a.n_items1 : sms, tcs::kThreads, tcs::kSmemBytes, st>>>(qa, k256, a);
+    FLOWMM_LAUNCHED("score_stats_tc");
+    const int n_negc = UH * a.GWpad;
+    score_combine_kernel<<<(n_negc + 255) / 256, 256, 0, st>>>(a.row_part, a.n_chunk, a.GW, a.GWpad, UH, a.negc);
+    FLOWMM_LAUNCHED("score_combine");
+    score_colsum_tc_kernel<<<a.n_items2 < sms ? a.n_items2 : sms, tcs::kThreads, tcs::kSmemBytes, st>>>(k128, qb, a);
+    FLOWMM_LAUNCHED("score_colsum_tc");
+    const int n = p.n_units * p.n_q_heads;
+    cross_mass_reduce<<<(n + 255) / 256, 256, 0, st>>>(a.cross_part, a.n_rt * 4, n, cross_mass);
+    FLOWMM_LAUNCHED("cross_mass_reduce");
+    return FLOWMM_OK;
+}
+
 flowmm_status run_score(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
                         float *importance, float *cross_mass, void *ws, cudaStream_t st) {
+    if (use_tc_score(p)) return run_score_tc(p, y, q, k, mod, importance, cross_mass, ws, st);
     ScoreArgs a;
     a.q = q; a.k = k; a.modality = mod; a.importance = importance;
     a.row_part = at<float2>(ws, y.row_part);
@@ -207,9 +273,6 @@ flowmm_status run_select(const flowmm_params &p, const float *importance, int32_
     return FLOWMM_OK;
 }
 
-bool use_tc(const flowmm_params &p) {
-    return p.path == FLOWMM_PATH_AUTO && p.dtype == FLOWMM_BF16 && p.head_dim == 128;
-}
 
 flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
                            const uint8_t *mod, const int32_t *retained, const int32_t *evicted,
@@ -230,20 +293,21 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     CUtensorMap k_map, cand_map;
     const uint64_t kd[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
     const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
-    const uint64_t cd[3] = {128, (uint64_t)y.c_tot, (uint64_t)UH};
-    const uint64_t cs[2] = {256, (uint64_t)y.c_tot * 256};
-    if (!tc::make_bf16_map(&k_map, k, 4, kd, ks, kMtRows) || !tc::make_bf16_map(&cand_map, g.cand_k, 3, cd, cs, kMtCols))
+    const uint64_t cd[4] = {128, (uint64_t)y.c_tot, (uint64_t)UH, 1};
+    const uint64_t cs[3] = {256, (uint64_t)y.c_tot * 256, (uint64_t)y.c_tot * 256 * (uint64_t)UH};
+    const uint32_t box_a[4] = {64, kMtRows, 1, 1}, box_b[4] = {64, kMtCols, 1, 1};
+    if (!tc::make_bf16_map(&k_map, k, 4, kd, ks, box_a) || !tc::make_bf16_map(&cand_map, g.cand_k, 4, cd, cs, box_b))
         return FLOWMM_ERR_CUDA;
     MatchTcArgs a;
     a.cand_count = g.cand_count; a.cand_slot = g.cand_slot; a.rank = g.rank; a.strategy = strategy;
     a.cand_scale = g.cand_scale; a.rn = g.rn; a.modality = mod; a.tile_mod = g.tile_mod;
     a.match = match; a.match_sim = match_sim; a.status = at<int>(ws, y.status);
     a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.E = E; a.Ctot = y.c_tot; a.n_rt = y.n_rt; a.n_items = UH * y.n_rt;
-    if (cudaFuncSetAttribute(match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMtSmemBytes) !=
+    if (cudaFuncSetAttribute(match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tcs::kSmemBytes) !=
         cudaSuccess)
         return FLOWMM_ERR_CUDA;
     const int grid = a.n_items < tc::sm_count() ? a.n_items : tc::sm_count();
-    match_tc_kernel<<<grid, kMtThreads, kMtSmemBytes, st>>>(k_map, cand_map, a);
+    match_tc_kernel<<<grid, tcs::kThreads, tcs::kSmemBytes, st>>>(k_map, cand_map, a);
     FLOWMM_LAUNCHED("match_tc");
     return FLOWMM_OK;
 }

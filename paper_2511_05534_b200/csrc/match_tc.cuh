@@ -11,20 +11,12 @@
 // An intra-modal layer visits only the candidate group of the row tile's modality.
 #pragma once
 #include "common.cuh"
-#include "tc_common.cuh"
+#include "tc_stream.cuh"
 
 namespace flowmm {
 
-constexpr int kMtRows = 128;                 // tokens per row tile (UMMA M)
-constexpr int kMtCols = 256;                 // candidates per column tile (UMMA N)
-constexpr int kMtThreads = 192;              // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
-constexpr uint32_t kMtABytes = kMtRows * 128 * 2;     // one row tile, both K halves
-constexpr uint32_t kMtBBytes = kMtCols * 128 * 2;
-constexpr uint32_t kMtSmemA = 0;
-constexpr uint32_t kMtSmemB = 2 * kMtABytes;
-constexpr uint32_t kMtSmemWin = kMtSmemB + 2 * kMtBBytes;
-constexpr uint32_t kMtSmemBar = kMtSmemWin + kMtRows * 32 * 4;
-constexpr uint32_t kMtSmemBytes = kMtSmemBar + 256 + 1024;   // + slack to align the base to 1024
+constexpr int kMtRows = tcs::kRows;          // tokens per row tile
+constexpr int kMtCols = tcs::kCols;          // candidates per column tile
 
 struct MatchPrepArgs {
     const void *k;
@@ -121,10 +113,13 @@ struct MatchTcArgs {
 };
 
 struct MatchItem {
-    int u, h, uh, rt, lo, hi, n_tiles, n_text, t0, n_vis;
+    int u, h, uh, rt, lo, hi, n_text, t0, n_vis;
     bool intra;
+    tcs::TilePlan tp;
 };
 
+// Which candidate columns a row tile has to visit: everything in a cross-modal layer or when the
+// tile mixes modalities, otherwise only the group of the tile's modality.
 __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) {
     MatchItem p;
     p.uh = item / A.n_rt; p.rt = item % A.n_rt;
@@ -137,111 +132,29 @@ __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) 
     if (!p.intra || tm == 3) { p.lo = 0; p.hi = end_all; }
     else if (tm == 1) { p.lo = 0; p.hi = p.n_text; }
     else { p.lo = p.t0; p.hi = p.t0 + p.n_vis; }
-    p.n_tiles = p.hi > p.lo ? (p.hi - p.lo + kMtCols - 1) / kMtCols : 0;
+    const int cols = p.hi > p.lo ? p.hi - p.lo : 0;
+    p.tp.a1 = p.rt * kMtRows; p.tp.a2 = p.h; p.tp.a3 = p.u;
+    p.tp.b1 = p.lo; p.tp.b2 = p.uh; p.tp.b3 = 0;
+    p.tp.step1 = kMtCols; p.tp.step2 = 0;
+    p.tp.n_tiles = (cols + kMtCols - 1) / kMtCols;
+    p.tp.cols_total = cols;
     return p;
 }
 
-// Persistent kernel: CTA b handles row-tile items b, b + gridDim.x, ...  One CTA per SM.
-__global__ void __launch_bounds__(kMtThreads, 1)
+// Persistent kernel, one CTA per SM; item = (unit, head, tile of 128 tokens).
+__global__ void __launch_bounds__(tcs::kThreads, 1)
 match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap cand_map,
                 const MatchTcArgs A) {
     extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *gen = smem_raw + (base - tc::smem_u32(smem_raw));
-    float *win = reinterpret_cast<float *>(gen + kMtSmemWin);
-    const uint32_t bars = base + kMtSmemBar;
-    // barrier slots: 0-1 a_full, 2-3 a_empty, 4-5 b_full, 6-7 b_empty, 8-9 t_full, 10-11 t_empty
-    auto bar = [&](int i) { return bars + 8u * i; };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(gen + kMtSmemBar + 128);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(gen + kMtSmemBar + 132);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < 10; ++i) tc::mbar_init(bar(i), 1);
-        tc::mbar_init(bar(10), 4);
-        tc::mbar_init(bar(11), 4);
-        *abort_flag = 0;
-        tc::mbar_init_fence();
-        tc::tma_prefetch_desc(&k_map);
-        tc::tma_prefetch_desc(&cand_map);
-    }
-    if (warp == 1) tc::tmem_alloc(tc::smem_u32(tmem_slot), 512);
-    tc::tc_fence_before();
-    __syncthreads();
-    tc::tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    if (warp == 0) {
-        if (lane == 0) {                                             // ---- TMA producer
-            int it = 0, bt = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
-                const MatchItem p = match_plan(A, item);
-                if (p.n_tiles == 0) continue;
-                const int sa = it & 1;
-                ok = tc::mbar_wait(bar(2 + sa), ((it >> 1) & 1) ^ 1, abort_flag, A.status);
-                if (!ok) break;
-                tc::mbar_expect_tx(bar(sa), kMtABytes);
-                const uint32_t a_dst = base + kMtSmemA + sa * kMtABytes;
-                tc::tma_load_4d(a_dst, &k_map, bar(sa), 0, p.rt * kMtRows, p.h, p.u);
-                tc::tma_load_4d(a_dst + kMtABytes / 2, &k_map, bar(sa), 64, p.rt * kMtRows, p.h, p.u);
-                for (int t = 0; t < p.n_tiles; ++t, ++bt) {
-                    const int sb = bt & 1;
-                    ok = tc::mbar_wait(bar(6 + sb), ((bt >> 1) & 1) ^ 1, abort_flag, A.status);
-                    if (!ok) break;
-                    tc::mbar_expect_tx(bar(4 + sb), kMtBBytes);
-                    const uint32_t b_dst = base + kMtSmemB + sb * kMtBBytes;
-                    tc::tma_load_3d(b_dst, &cand_map, bar(4 + sb), 0, p.lo + t * kMtCols, p.uh);
-                    tc::tma_load_3d(b_dst + kMtBBytes / 2, &cand_map, bar(4 + sb), 64, p.lo + t * kMtCols, p.uh);
-                }
-                ++it;
-            }
-            if (!ok) {                                               // let copies already issued land
-                for (int i = 0; i < 2; ++i) {
-                    for (int spin = 0; spin < (1 << 16) && !tc::mbar_try_wait(bar(i), 0) && !tc::mbar_try_wait(bar(i), 1); ++spin) {}
-                    for (int spin = 0; spin < (1 << 16) && !tc::mbar_try_wait(bar(4 + i), 0) && !tc::mbar_try_wait(bar(4 + i), 1); ++spin) {}
-                }
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0) {                                             // ---- MMA issuer
-            int it = 0, bt = 0, tt = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
-                const MatchItem p = match_plan(A, item);
-                if (p.n_tiles == 0) continue;
-                const int sa = it & 1;
-                ok = tc::mbar_wait(bar(sa), (it >> 1) & 1, abort_flag, A.status);
-                if (!ok) break;
-                const uint32_t a_base = base + kMtSmemA + sa * kMtABytes;
-                for (int t = 0; t < p.n_tiles; ++t, ++bt, ++tt) {
-                    const int sb = bt & 1, ta = tt & 1;
-                    ok = tc::mbar_wait(bar(4 + sb), (bt >> 1) & 1, abort_flag, A.status) &&
-                         tc::mbar_wait(bar(10 + ta), ((tt >> 1) & 1) ^ 1, abort_flag, A.status);
-                    if (!ok) break;
-                    tc::tc_fence_after();
-                    const int ncols = min(kMtCols, p.hi - (p.lo + t * kMtCols));
-                    const uint32_t idesc = tc::idesc_bf16(kMtRows, (uint32_t)((ncols + 15) & ~15));
-                    const uint32_t b_base = base + kMtSmemB + sb * kMtBBytes;
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {                 // 8 K slices of 16 elements
-                        const uint32_t a_off = (ks >> 2) * (kMtABytes / 2) + (ks & 3) * 32;
-                        const uint32_t b_off = (ks >> 2) * (kMtBBytes / 2) + (ks & 3) * 32;
-                        tc::umma_bf16(tmem_base + ta * kMtCols, tc::smem_desc_sw128(a_base, a_off),
-                                      tc::smem_desc_sw128(b_base, b_off), idesc, ks > 0);
-                    }
-                    tc::umma_commit(bar(6 + sb));                    // B stage free once these MMAs are done
-                    tc::umma_commit(bar(8 + ta));                    // accumulator ready
-                }
-                if (!ok) break;
-                tc::umma_commit(bar(2 + sa));                        // A stage free
-                ++it;
-            }
-        }
-    } else {                                                         // ---- epilogue warps
-        const int quarter = warp & 3;                                // TMEM lanes this warp may read
-        const int row = quarter * 32 + lane;
-        float4 *wrow = reinterpret_cast<float4 *>(win + row * 32);
+    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &cand_map);
+    auto plan = [&](int item) { return match_plan(A, item).tp; };
+    if (c.warp == 0) {
+        if (c.lane == 0) tcs::producer(c, &k_map, &cand_map, A.n_items, tcs::kAStage, tcs::kBStage, plan, A.status);
+    } else if (c.warp == 1) {
+        if (c.lane == 0) tcs::mma_issuer(c, A.n_items, plan, A.status);
+    } else {
+        const int lane = c.lane, row = (c.warp & 3) * 32 + lane;
+        float4 *wrow = reinterpret_cast<float4 *>(c.epi_scratch()) + row * 8;   // 32 floats per row
         int tt = 0;
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
@@ -255,20 +168,18 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             float best = -INFINITY;
             int best_cc = -1;
             const float *scale = A.cand_scale + (int64_t)p.uh * A.Ctot;
-            for (int t = 0; ok && t < p.n_tiles; ++t, ++tt) {
-                const int ta = tt & 1;
-                ok = tc::mbar_wait(bar(8 + ta), (tt >> 1) & 1, abort_flag, A.status);
+            for (int t = 0; ok && t < p.tp.n_tiles; ++t, ++tt) {
+                ok = tcs::acc_wait(c, tt, A.status);
                 if (!ok) break;
-                tc::tc_fence_after();
                 const int col0 = p.lo + t * kMtCols;
                 const int ncols = min(kMtCols, p.hi - col0);
-                for (int c = 0; c * 32 < ncols; ++c) {
-                    const int cc = col0 + c * 32;
+                for (int ch = 0; ch * 32 < ncols; ++ch) {
+                    const int cc = col0 + ch * 32;
                     const bool full = (cc + 32 <= r1hi) || (cc >= r2lo && cc + 32 <= r2hi);
                     const bool none = !((cc < r1hi) || (cc + 32 > r2lo && cc < r2hi));
                     if (__all_sync(0xFFFFFFFFu, none)) continue;
                     uint32_t acc[32];
-                    tc::tmem_ld32(tmem_base + ta * kMtCols + c * 32 + ((uint32_t)(quarter * 32) << 16), acc);
+                    tc::tmem_ld32(tcs::acc_addr(c, tt, ch), acc);
                     const float4 *sp = reinterpret_cast<const float4 *>(scale + cc);
                     float4 s4[8];
 #pragma unroll
@@ -305,9 +216,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                             wrow[q4 ^ (row & 7)] = make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
                     }
                 }
-                tc::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(bar(10 + ta));
+                tcs::acc_release(c, tt);
             }
             if (!ok) break;
             if (in_range) {
@@ -318,7 +227,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     if (best_cc >= 0) {
                         int idx = 0;
 #pragma unroll
-                        for (int q4 = 7; q4 >= 0; --q4) {
+                        for (int q4 = 7; q4 >= 0; --q4) {            // lowest column that holds the maximum
                             const float4 w = wrow[q4 ^ (row & 7)];
                             if (w.w == best) idx = 4 * q4 + 3;
                             if (w.z == best) idx = 4 * q4 + 2;
@@ -334,10 +243,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             }
         }
     }
-    tc::tc_fence_before();
-    __syncthreads();
-    tc::tc_fence_after();
-    if (warp == 1) tc::tmem_dealloc(tmem_base, 512);
+    tcs::teardown(c);
 }
 
 }  // namespace flowmm

@@ -24,19 +24,17 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// bf16 tensor of `rank` dims (innermost first, contiguous innermost), box of 64 elements x
-// `box_rows` rows, 128-byte swizzle, zero fill outside the tensor.  strides_bytes[i] is the
-// stride of dim i+1.  Returns false if the driver rejects the description.
+// bf16 tensor of `rank` dims (innermost first, contiguous innermost), box as given (box[0] = 64
+// elements = one 128-byte swizzle span), 128-byte swizzle, zero fill outside the tensor.
+// strides_bytes[i] is the stride of dim i+1.  Returns false if the driver rejects the description.
 inline bool make_bf16_map(CUtensorMap *map, const void *base, int rank, const uint64_t *dims,
-                          const uint64_t *strides_bytes, uint32_t box_rows) {
+                          const uint64_t *strides_bytes, const uint32_t *box_dims) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t gdim[5], gstride[4];
     cuuint32_t box[5], estr[5];
-    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; box[i] = 1; estr[i] = 1; }
+    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; box[i] = box_dims[i]; estr[i] = 1; }
     for (int i = 0; i + 1 < rank; ++i) gstride[i] = strides_bytes[i];
-    box[0] = 64;
-    box[1] = box_rows;
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gdim, gstride, box,
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
