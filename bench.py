@@ -39,6 +39,7 @@ def parse_args():
                     help="retention budget in 1/1000 of the context (0: 100 if the workload lists it, else its first)")
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers (0 = the whole stack)")
     ap.add_argument("--path", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--sets", type=int, default=0, help="rotating input sets held on the device (0 = automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-units", type=int, default=0)
     return ap.parse_args()
@@ -238,6 +239,8 @@ def run_ours(args):
     n_sets = max(2, min(8, int(1.5e9 // max(1, bytes_per_set)) + 1))
     if bytes_per_set > 20e9:
         n_sets = 1            # a set this large cannot stay in the 126 MB L2 anyway
+    if args.sets > 0:
+        n_sets = args.sets
     sets = [inputs.make_stack_device(wl, dev, units, seed_offset=rank * 100 + i) for i in range(n_sets)]
     k_out = torch.empty((U, wl.n_kv_heads, B, wl.head_dim), dtype=sets[0][1].dtype, device=dev)
     v_out = torch.empty_like(k_out)
