@@ -211,7 +211,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2511_05534_b200 import binding as F
-    from paper_2511_05534_b200 import build, configs, inputs
+    from paper_2511_05534_b200 import build, configs, inputs, shard
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -225,7 +225,7 @@ def run_ours(args):
 
     wl = configs.get(args.workload)
     n_layers = args.layers if args.layers > 0 else wl.n_layers
-    units = [(l, s) for l in range(n_layers) for s in range(wl.n_seqs)]
+    units = shard.rank_units(n_layers, wl.n_seqs, rank, world)
     U = len(units)
     B = wl.n_keep(args.permille)
     dt_code = F.BF16 if wl.dtype == "bf16" else F.F32
@@ -241,7 +241,7 @@ def run_ours(args):
         n_sets = 1            # a set this large cannot stay in the 126 MB L2 anyway
     if args.sets > 0:
         n_sets = args.sets
-    sets = [inputs.make_stack_device(wl, dev, units, seed_offset=rank * 100 + i) for i in range(n_sets)]
+    sets = [inputs.make_stack_device(wl, dev, units, seed_offset=shard.seed_offset(rank, i)) for i in range(n_sets)]
     k_out = torch.empty((U, wl.n_kv_heads, B, wl.head_dim), dtype=sets[0][1].dtype, device=dev)
     v_out = torch.empty_like(k_out)
     ws = F.alloc_workspace(p, dev)
@@ -274,13 +274,10 @@ def run_ours(args):
     status = F.flowmm_last_device_status(ws)
     if status != 0:
         raise RuntimeError("device status: " + F.status_string(status))
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = shard.max_over_ranks(ms_total, dev)
     ms_step = ms_total / args.steps
     tokens_layers = wl.n_seqs * wl.seq_len * n_layers        # tokens x layers compressed per step per GPU
-    value = world * tokens_layers / (ms_step * 1e-3)
+    value = shard.aggregate_throughput(tokens_layers, world, ms_step)
 
     # per-kernel attribution: the same steps again with an event after every kernel
     F.flowmm_profile_enable(True)
@@ -337,11 +334,8 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * tokens_layers / (e2e_ms / e2e_steps * 1e-3)
+    e2e_ms = shard.max_over_ranks(e2e_ms, dev)
+    e2e_value = shard.aggregate_throughput(tokens_layers, world, e2e_ms / e2e_steps)
 
     if rank == 0:
         line = {
