@@ -152,6 +152,33 @@ flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v,
                            void *k_out, void *v_out, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * flowmm_merge without a caller-provided workspace.  (The paper has no counterpart: this is a
+ * packaging variant of step 5 for callers that cannot allocate device memory - a plugin running
+ * inside another runtime's memory pool, code running while that pool is frozen, a host that is
+ * handed fixed buffers only.  They still pass the inputs and the two output tensors; what they
+ * cannot provide is the scratch flowmm_merge needs for its slot lists and partial sums.)
+ *
+ * The scratch is a fixed array of FLOWMM_MERGE_STATIC_BYTES inside the library image; every GPU
+ * that loads the library holds one copy until the process exits.  The call makes no cudaMalloc
+ * or cudaFree and calls no allocating routine.  Arguments, outputs and results are those of
+ * flowmm_merge (same kernels, same fixed accumulation order, so the outputs are bit-identical).
+ *
+ * Limits and rules:
+ *   - The scratch a problem needs is about 8 E + 12 (B + 1) bytes per (unit, KV head) plus
+ *     (2 E / 64 + 2) * (8 head_dim + 16) bytes per (unit, KV head) of partial sums; if that
+ *     exceeds the array the call returns FLOWMM_ERR_WORKSPACE and launches nothing.
+ *   - The first call on a device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents;
+ *     nothing in it needs clearing between calls.  Two calls that overlap on the GPU (different
+ *     streams, or graphs replayed concurrently) race on it: keep them ordered.
+ */
+#define FLOWMM_MERGE_STATIC_BYTES (8u << 20)
+flowmm_status flowmm_merge_static(const flowmm_params *p, const void *k, const void *v, const int32_t *retained_idx,
+                                  const int32_t *evicted_idx, const int32_t *match, const float *match_sim,
+                                  void *k_out, void *v_out, void *cuda_stream);
+
+/*
  * Steps 1-5 in order on one stream: the whole per-layer FlowMM compression of Section 3.3.
  * The diagnostic outputs (importance ... match_sim, layouts as above) may each be NULL, in
  * which case the intermediate lives in the workspace only.

@@ -28,7 +28,7 @@ PATH_AUTO, PATH_SIMT = 0, 1
 EXPORTS = (
     "flowmm_workspace_bytes", "flowmm_score", "flowmm_layer_flow", "flowmm_select", "flowmm_match", "flowmm_merge",
     "flowmm_compress_layer", "flowmm_last_device_status", "flowmm_last_launch_count", "flowmm_status_string",
-    "flowmm_profile_enable", "flowmm_profile_read",
+    "flowmm_profile_enable", "flowmm_profile_read", "flowmm_merge_static",
 )
 
 
@@ -118,6 +118,7 @@ def load() -> ctypes.CDLL:
         lib.flowmm_profile_read.restype = ctypes.c_int32
         for name in EXPORTS[:8]:
             getattr(lib, name).restype = ctypes.c_int
+        lib.flowmm_merge_static.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -191,6 +192,14 @@ def flowmm_merge(p: Params, k, v, retained_idx, evicted_idx, match, match_sim, k
     _check(load().flowmm_merge(ctypes.byref(cp), _p(k), _p(v), _p(retained_idx), _p(evicted_idx), _p(match),
                                _p(match_sim), _p(k_out), _p(v_out), _p(ws), ctypes.c_size_t(ws.numel()), _stream()),
            "flowmm_merge")
+
+
+def flowmm_merge_static(p: Params, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out):
+    """flowmm_merge for callers that cannot allocate: no workspace argument, the scratch is a
+    fixed array inside the library (see include/flowmm.h for its size limit and sharing rules)."""
+    cp = p.c(k=k, v=v, ko=k_out, vo=v_out)
+    _check(load().flowmm_merge_static(ctypes.byref(cp), _p(k), _p(v), _p(retained_idx), _p(evicted_idx), _p(match),
+                                      _p(match_sim), _p(k_out), _p(v_out), _stream()), "flowmm_merge_static")
 
 
 def flowmm_compress_layer(p: Params, q_win, k, v, modality, k_out, v_out, ws, importance=None, rho=None,

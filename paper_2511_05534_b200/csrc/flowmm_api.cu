@@ -6,6 +6,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "match_tc.cuh"
 #include "score_tc.cuh"
@@ -552,3 +554,76 @@ const char *flowmm_status_string(flowmm_status s) {
 }
 
 }  // extern "C"
+
+// ---- merge without caller scratch --------------------------------------------------------------
+// Scratch of flowmm_merge_static: lives in the library image, one copy per GPU that loads it.
+static __device__ __align__(256) unsigned char g_merge_static_scratch[FLOWMM_MERGE_STATIC_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices] = {};          // device address of the array, per device ordinal
+
+// The array's name is only a handle in host code; the address a kernel can use comes from the
+// runtime, once per device, with that device current.
+flowmm_status merge_static_base(void **base) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return FLOWMM_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_merge_static_scratch) != cudaSuccess || !ptr) return FLOWMM_ERR_CUDA;
+        g_static_ptr[dev] = ptr;
+    }
+    *base = g_static_ptr[dev];
+    return FLOWMM_OK;
+}
+
+// The part of the workspace layout that the merge step touches, packed from offset 0.
+Layout make_merge_layout(const flowmm_params &p) {
+    Layout y = {};
+    const size_t UH = (size_t)p.n_units * p.n_kv_heads, B = p.n_keep, E = (size_t)p.seq_len - B, D = p.head_dim;
+    y.max_pieces = (int)(B + E / kPiece + 1);
+    y.max_parts = (int)(2 * (E / kPiece) + 2);
+    y.csr_passes = 1;
+    while (y.csr_passes < 4 && (B >> (8 * y.csr_passes)) != 0) ++y.csr_passes;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { const size_t at = o; o += align256(bytes); return at; };
+    y.sort_a = take(UH * E * 4);
+    y.sort_b = take(UH * E * 4);
+    y.off = take(UH * (B + 1) * 4);
+    y.piece_off = take(UH * (B + 1) * 4);
+    y.part_off = take(UH * (B + 1) * 4);
+    y.partial = take(UH * (size_t)y.max_parts * (2 * D + 4) * 4);
+    y.total = o;
+    return y;
+}
+
+}  // namespace
+
+extern "C" flowmm_status flowmm_merge_static(const flowmm_params *p, const void *k, const void *v,
+                                             const int32_t *retained_idx, const int32_t *evicted_idx,
+                                             const int32_t *match, const float *match_sim, void *k_out, void *v_out,
+                                             void *cuda_stream) {
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
+    FLOWMM_TRY(validate(p));
+    const bool has_e = p->n_keep < p->seq_len;
+    if (!k || !v || !retained_idx || !k_out || !v_out) return FLOWMM_ERR_NULL;
+    if (has_e && (!evicted_idx || !match || !match_sim)) return FLOWMM_ERR_NULL;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out) ||
+        !strides_ok(p->k_stride, p->head_dim) || !strides_ok(p->v_stride, p->head_dim) ||
+        !strides_ok(p->ko_stride, p->head_dim) || !strides_ok(p->vo_stride, p->head_dim))
+        return FLOWMM_ERR_ALIGN;
+    const Layout y = make_merge_layout(*p);
+    if (y.total > (size_t)FLOWMM_MERGE_STATIC_BYTES) return FLOWMM_ERR_WORKSPACE;   // problem too large for the array
+    FLOWMM_TRY(check_device());
+    void *base = nullptr;
+    FLOWMM_TRY(merge_static_base(&base));
+    // Nothing in this scratch has to start at zero: the CSR arrays are written in full before they
+    // are read and a partial-sum record is only read for pieces that wrote it in the same call.
+    return run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, base,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
