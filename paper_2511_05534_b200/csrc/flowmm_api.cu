@@ -94,18 +94,26 @@ Layout make_layout(const flowmm_params &p) {
     y.evicted = take(U * Hkv * E * 4);
     y.match = take(U * Hkv * E * 4);
     y.match_sim = take(U * Hkv * E * 4);
-    y.n_rt = (int)((L + tcs::kRows - 1) / tcs::kRows);
-    {   // pass 1 of the tensor-core scoring: key chunks of whole 256-key tiles
-        y.tc_n_qt = (int)((G * W + tcs::kRows - 1) / tcs::kRows);
+    y.n_rt = (int)((L + tcs::kItemRows - 1) / tcs::kItemRows);
+    {   // pass 1 of the tensor-core scoring: key chunks of whole 256-key tiles, sized so that the
+        // persistent CTAs (one per SM, 148 on B200) finish their last round together
+        y.tc_n_qt = (int)((G * W + tcs::kItemRows - 1) / tcs::kItemRows);
         const int key_tiles = (int)((L + tcs::kCols - 1) / tcs::kCols);
-        int want = (int)((2 * 148 + U * Hkv * y.tc_n_qt - 1) / (U * Hkv * y.tc_n_qt));
-        want = want < 1 ? 1 : (want > key_tiles ? key_tiles : want);
-        y.tc_tiles_per_chunk = (key_tiles + want - 1) / want;
+        const long base_items = (long)(U * Hkv) * y.tc_n_qt;
+        double best_cost = 1e300;
+        y.tc_tiles_per_chunk = key_tiles;
+        for (int want = 1; want <= key_tiles; ++want) {
+            const int tpc = (key_tiles + want - 1) / want;
+            const int nc = (key_tiles + tpc - 1) / tpc;
+            const long rounds = (base_items * nc + 147) / 148;
+            const double cost = (double)rounds * (tpc + 0.75);     // 0.75 tile: per-item start-up
+            if (cost < best_cost - 1e-9) { best_cost = cost; y.tc_tiles_per_chunk = tpc; }
+        }
         y.tc_n_chunk = (key_tiles + y.tc_tiles_per_chunk - 1) / y.tc_tiles_per_chunk;
         y.gw_pad = (int)((G * W + tcs::kCols - 1) / tcs::kCols * tcs::kCols);
     }
     const size_t max_chunk1 = (size_t)(y.n_chunk1 > y.tc_n_chunk ? y.n_chunk1 : y.tc_n_chunk);
-    const size_t max_chunk2 = (size_t)(y.n_chunk2 > 4 * y.n_rt ? y.n_chunk2 : 4 * y.n_rt);
+    const size_t max_chunk2 = (size_t)(y.n_chunk2 > 8 * y.n_rt ? y.n_chunk2 : 8 * y.n_rt);
     y.row_part = take(U * Hq * W * max_chunk1 * 8);
     y.cross_part = take(U * Hq * max_chunk2 * 4);
     y.negc = take(U * Hkv * (size_t)y.gw_pad * 4);
@@ -118,7 +126,7 @@ Layout make_layout(const flowmm_params &p) {
     y.partial = take(U * Hkv * (size_t)y.max_parts * (2 * D + 4) * 4);
     y.c_tot = (int)((B + 31) / 32 * 32 + 32);
     y.cand_k = take(U * Hkv * (size_t)y.c_tot * 128 * 2);
-    y.cand_scale = take(U * Hkv * (size_t)y.c_tot * 4);
+    y.cand_scale = take(U * Hkv * (size_t)y.c_tot * 4 + 1024);   // + one tile of slack: whole 256-column slices are copied
     y.cand_slot = take(U * Hkv * (size_t)y.c_tot * 4);
     y.cand_count = take(U * Hkv * 2 * 4);
     y.rank = take(U * Hkv * L * 4);
@@ -190,7 +198,7 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     a.importance = importance; a.cross_part = at<float>(ws, y.cross_part); a.status = at<int>(ws, y.status);
     a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.G = G; a.W = W; a.L = p.seq_len; a.GW = G * W; a.GWpad = y.gw_pad;
     a.n_qt = y.tc_n_qt; a.n_chunk = y.tc_n_chunk; a.tiles_per_chunk = y.tc_tiles_per_chunk; a.n_rt = y.n_rt;
-    a.a_heads = G < tcs::kRows / W ? G : tcs::kRows / W;
+    a.a_heads = G < tcs::kRows / W ? G : tcs::kRows / W;        // one A half holds 128 proxy rows
     a.b_heads = G < tcs::kCols / W ? G : tcs::kCols / W;
     a.n_items1 = UH * a.n_qt * a.n_chunk; a.n_items2 = UH * a.n_rt;
     const float scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.f / sqrtf((float)p.head_dim);
@@ -220,7 +228,7 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     score_colsum_tc_kernel<<<a.n_items2 < sms ? a.n_items2 : sms, tcs::kThreads, tcs::kSmemBytes, st>>>(k128, qb, a);
     FLOWMM_LAUNCHED("score_colsum_tc");
     const int n = p.n_units * p.n_q_heads;
-    cross_mass_reduce<<<(n + 255) / 256, 256, 0, st>>>(a.cross_part, a.n_rt * 4, n, cross_mass);
+    cross_mass_reduce<<<(n + 255) / 256, 256, 0, st>>>(a.cross_part, a.n_rt * 8, n, cross_mass);
     FLOWMM_LAUNCHED("cross_mass_reduce");
     return FLOWMM_OK;
 }

@@ -3,7 +3,7 @@
 // Per (unit, KV head) the admissible pivots (importance <= tau) are gathered into a dense
 // candidate matrix, text candidates first and visual candidates from the next multiple of 32.
 // The similarity contraction then runs as  S[128 tokens x 256 candidates] = K_tile . C_tile^T
-// on tcgen05 with the token rows taken straight from the caller's K by TMA (every token of the
+// (two such 128-token halves per candidate tile) on tcgen05 with the token rows taken straight from the caller's K by TMA (every token of the
 // head in prompt order; rows that are pivots are computed and dropped), fp32 accumulators in
 // TMEM, and an epilogue that scales each column by the candidate's reciprocal norm and keeps a
 // running row maximum.  Raw bf16 keys feed the MMA (their products are exact in fp32); the
@@ -15,7 +15,8 @@
 
 namespace flowmm {
 
-constexpr int kMtRows = tcs::kRows;          // tokens per row tile
+constexpr int kMtRows = tcs::kRows;          // tokens per accumulator half
+constexpr int kMtItemRows = tcs::kItemRows;  // tokens per item (two halves)
 constexpr int kMtCols = tcs::kCols;          // candidates per column tile
 
 struct MatchPrepArgs {
@@ -28,7 +29,7 @@ struct MatchPrepArgs {
     int *cand_slot;              // [UH, Ctot]
     int *cand_count;             // [UH, 2]  admissible text / visual pivots
     int *rank;                   // [UH, L]  position in the non-pivot list, or -1 for a pivot
-    uint8_t *tile_mod;           // [U, n_rt] bit 0: tile holds text tokens, bit 1: visual tokens
+    uint8_t *tile_mod;           // [U, n_rt] per tile of 256 tokens; bit 0: holds text tokens, bit 1: visual tokens
     int Hkv, L, B, E, Ctot, n_rt;
     float tau_eff;
     int64_t ks[3];
@@ -48,14 +49,14 @@ __global__ void __launch_bounds__(256) match_prepare_kernel(const MatchPrepArgs 
     int *slot_out = A.cand_slot + (int64_t)uh * A.Ctot;
     float *scale_out = A.cand_scale + (int64_t)uh * A.Ctot;
 
-    for (int i = tid; i < A.Ctot; i += blockDim.x) { slot_out[i] = -1; scale_out[i] = 0.f; }
+    for (int i = tid; i < A.Ctot; i += blockDim.x) { slot_out[i] = -1; scale_out[i] = __int_as_float(0x7FC00000); }   // NaN: no candidate here
     for (int s = tid; s < A.B; s += blockDim.x) rank[ret[s]] = -1;
     for (int j = tid; j < A.E; j += blockDim.x) rank[evi[j]] = j;
     if (h == 0) {
         for (int t = tid; t < A.n_rt; t += blockDim.x) {
             int bits = 0;
-            const int hi = min(A.L, (t + 1) * kMtRows);
-            for (int i = t * kMtRows; i < hi; ++i) bits |= mod[i] ? 2 : 1;
+            const int hi = min(A.L, (t + 1) * kMtItemRows);
+            for (int i = t * kMtItemRows; i < hi; ++i) bits |= mod[i] ? 2 : 1;
             A.tile_mod[(int64_t)u * A.n_rt + t] = (uint8_t)bits;
         }
     }
@@ -114,12 +115,12 @@ struct MatchTcArgs {
 
 struct MatchItem {
     int u, h, uh, rt, lo, hi, n_text, t0, n_vis;
-    bool intra;
+    bool intra, mixed;
     tcs::TilePlan tp;
 };
 
-// Which candidate columns a row tile has to visit: everything in a cross-modal layer or when the
-// tile mixes modalities, otherwise only the group of the tile's modality.
+// Which candidate columns a tile of 256 tokens has to visit: everything in a cross-modal layer or
+// when the tile mixes modalities, otherwise only the group of the tile's modality.
 __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) {
     MatchItem p;
     p.uh = item / A.n_rt; p.rt = item % A.n_rt;
@@ -128,95 +129,101 @@ __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) 
     p.t0 = (p.n_text + 31) & ~31;
     p.intra = A.strategy[p.u] == 0;
     const int tm = A.tile_mod[(int64_t)p.u * A.n_rt + p.rt];
+    p.mixed = tm == 3;
     const int end_all = p.n_vis > 0 ? p.t0 + p.n_vis : p.n_text;
     if (!p.intra || tm == 3) { p.lo = 0; p.hi = end_all; }
     else if (tm == 1) { p.lo = 0; p.hi = p.n_text; }
     else { p.lo = p.t0; p.hi = p.t0 + p.n_vis; }
     const int cols = p.hi > p.lo ? p.hi - p.lo : 0;
-    p.tp.a1 = p.rt * kMtRows; p.tp.a2 = p.h; p.tp.a3 = p.u;
+    p.tp.a1 = p.rt * kMtItemRows; p.tp.a2 = p.h; p.tp.a3 = p.u;
+    p.tp.h1 = kMtRows; p.tp.h2 = 0;
+    p.tp.n_halves = p.tp.a1 + kMtRows < A.L ? 2 : 1;
     p.tp.b1 = p.lo; p.tp.b2 = p.uh; p.tp.b3 = 0;
     p.tp.step1 = kMtCols; p.tp.step2 = 0;
     p.tp.n_tiles = (cols + kMtCols - 1) / kMtCols;
     p.tp.cols_total = cols;
+    p.tp.extra = A.cand_scale + (int64_t)p.uh * A.Ctot + p.lo;
     return p;
 }
 
-// Persistent kernel, one CTA per SM; item = (unit, head, tile of 128 tokens).
+// Persistent kernel, one CTA per SM; item = (unit, head, tile of 256 tokens).
 __global__ void __launch_bounds__(tcs::kThreads, 1)
 match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap cand_map,
                 const MatchTcArgs A) {
-    extern __shared__ uint8_t smem_raw[];
-    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &cand_map);
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &cand_map, A.status);
+    if (!c.ok) return;
     auto plan = [&](int item) { return match_plan(A, item).tp; };
     if (c.warp == 0) {
-        if (c.lane == 0) tcs::producer(c, &k_map, &cand_map, A.n_items, tcs::kAStage, tcs::kBStage, plan, A.status);
+        if (c.lane == 0) tcs::producer(c, &k_map, &cand_map, A.n_items, tcs::kAHalf, tcs::kBStage, plan, A.status);
     } else if (c.warp == 1) {
         if (c.lane == 0) tcs::mma_issuer(c, A.n_items, plan, A.status);
     } else {
-        const int lane = c.lane, row = (c.warp & 3) * 32 + lane;
-        float4 *wrow = reinterpret_cast<float4 *>(c.epi_scratch()) + row * 8;   // 32 floats per row
-        int tt = 0;
+        const int lane = c.lane, row = c.quarter * 32 + lane;
+        float4 *wrow = reinterpret_cast<float4 *>(c.epi_scratch()) + row * 4;   // 16 floats per row
+        int k = 0, bt = 0;
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
             const MatchItem p = match_plan(A, item);
-            const int token = p.rt * kMtRows + row;
+            const bool active = !p.tp.empty() && c.group < p.tp.n_halves;
+            const int token = p.rt * kMtItemRows + c.group * kMtRows + row;
             const bool in_range = token < A.L;
             const int my_mod = in_range ? A.modality[(int64_t)p.u * A.L + token] : 0;
-            int r1hi = p.n_text, r2lo = p.t0, r2hi = p.t0 + p.n_vis;     // this row's admissible columns
+            // admissible columns of this row; only consulted where rows of a tile differ (row_masked)
+            int r1hi = p.n_text, r2lo = p.t0, r2hi = p.t0 + p.n_vis;
             if (p.intra) { if (my_mod == 0) r2hi = r2lo; else r1hi = 0; }
-            if (!in_range) { r1hi = 0; r2hi = r2lo; }
+            const bool row_masked = p.intra && p.mixed;
             float best = -INFINITY;
             int best_cc = -1;
-            const float *scale = A.cand_scale + (int64_t)p.uh * A.Ctot;
-            for (int t = 0; ok && t < p.tp.n_tiles; ++t, ++tt) {
-                ok = tcs::acc_wait(c, tt, A.status);
-                if (!ok) break;
-                const int col0 = p.lo + t * kMtCols;
-                const int ncols = min(kMtCols, p.hi - col0);
-                for (int ch = 0; ch * 32 < ncols; ++ch) {
-                    const int cc = col0 + ch * 32;
-                    const bool full = (cc + 32 <= r1hi) || (cc >= r2lo && cc + 32 <= r2hi);
-                    const bool none = !((cc < r1hi) || (cc + 32 > r2lo && cc < r2hi));
-                    if (__all_sync(0xFFFFFFFFu, none)) continue;
-                    uint32_t acc[32];
-                    tc::tmem_ld32(tcs::acc_addr(c, tt, ch), acc);
-                    const float4 *sp = reinterpret_cast<const float4 *>(scale + cc);
-                    float4 s4[8];
+            if (!active) {
+                if (!p.tp.empty()) bt += p.tp.n_tiles;               // keep the B-tile count in step
+            } else {
+                for (int t = 0; ok && t < p.tp.n_tiles; ++t, ++k, ++bt) {
+                    const int col0 = p.lo + t * kMtCols;
+                    const int ncols = min(kMtCols, p.hi - col0);
+                    ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
+                    if (!ok) break;
+                    const float4 *scale4 = c.extra(bt);              // reciprocal norms of this tile's candidates
+                    tcs::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
+                        const int cc = col0 + ch * 32;
+                        float v[32];
 #pragma unroll
-                    for (int q4 = 0; q4 < 8; ++q4) s4[q4] = __ldg(sp + q4);
-                    tc::tmem_ld_wait();
-                    float v[32];
-#pragma unroll
-                    for (int q4 = 0; q4 < 8; ++q4) {
-                        v[4 * q4 + 0] = __uint_as_float(acc[4 * q4 + 0]) * s4[q4].x;
-                        v[4 * q4 + 1] = __uint_as_float(acc[4 * q4 + 1]) * s4[q4].y;
-                        v[4 * q4 + 2] = __uint_as_float(acc[4 * q4 + 2]) * s4[q4].z;
-                        v[4 * q4 + 3] = __uint_as_float(acc[4 * q4 + 3]) * s4[q4].w;
-                    }
-                    if (!__all_sync(0xFFFFFFFFu, full)) {            // ragged group edge or mixed-modality tile
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int col = cc + j;
-                            const bool valid = (col < r1hi) || (col >= r2lo && col < r2hi);
-                            v[j] = valid ? v[j] : -INFINITY;
+                        for (int q4 = 0; q4 < 8; ++q4) {     // a column that is no candidate has scale NaN and never wins
+                            const float4 s4 = scale4[ch * 8 + q4];
+                            v[4 * q4 + 0] = __uint_as_float(acc[4 * q4 + 0]) * s4.x;
+                            v[4 * q4 + 1] = __uint_as_float(acc[4 * q4 + 1]) * s4.y;
+                            v[4 * q4 + 2] = __uint_as_float(acc[4 * q4 + 2]) * s4.z;
+                            v[4 * q4 + 3] = __uint_as_float(acc[4 * q4 + 3]) * s4.w;
                         }
-                    }
-                    float m12[12];
+                        if (row_masked) {                    // intra-modal layer, tile with tokens of both modalities
 #pragma unroll
-                    for (int i = 0; i < 10; ++i) m12[i] = tc::max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-                    m12[10] = v[30]; m12[11] = v[31];
-                    const float a0 = tc::max3(m12[0], m12[1], m12[2]), a1 = tc::max3(m12[3], m12[4], m12[5]);
-                    const float a2 = tc::max3(m12[6], m12[7], m12[8]), a3 = tc::max3(m12[9], m12[10], m12[11]);
-                    const float cmax = fmaxf(tc::max3(a0, a1, a2), a3);
-                    if (cmax > best) {                               // strict: an earlier chunk keeps a tie
-                        best = cmax;
-                        best_cc = cc;
+                            for (int j = 0; j < 32; ++j) {
+                                const int col = cc + j;
+                                const bool valid = (col < r1hi) || (col >= r2lo && col < r2hi);
+                                v[j] = valid ? v[j] : -INFINITY;
+                            }
+                        }
+                        float lo5[5], hi5[5];
 #pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4)               // keep the chunk to find the column later
-                            wrow[q4 ^ (row & 7)] = make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
-                    }
+                        for (int i = 0; i < 5; ++i) {
+                            lo5[i] = tc::max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
+                            hi5[i] = tc::max3(v[16 + 3 * i], v[17 + 3 * i], v[18 + 3 * i]);
+                        }
+                        const float lo = tc::max3(tc::max3(lo5[0], lo5[1], lo5[2]), tc::max3(lo5[3], lo5[4], v[15]), -INFINITY);
+                        const float hi = tc::max3(tc::max3(hi5[0], hi5[1], hi5[2]), tc::max3(hi5[3], hi5[4], v[31]), -INFINITY);
+                        const float cmax = fmaxf(lo, hi);
+                        if (cmax > best) {                           // strict: an earlier chunk keeps a tie
+                            best = cmax;
+                            const bool low = lo >= hi;               // a tie between the halves goes to the lower columns
+                            best_cc = low ? cc : cc + 16;
+#pragma unroll
+                            for (int q4 = 0; q4 < 4; ++q4)           // keep the 16 columns to find the exact one later
+                                wrow[q4] = low ? make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3])
+                                               : make_float4(v[16 + 4 * q4], v[17 + 4 * q4], v[18 + 4 * q4], v[19 + 4 * q4]);
+                        }
+                    });
+                    tcs::acc_release(c);
                 }
-                tcs::acc_release(c, tt);
             }
             if (!ok) break;
             if (in_range) {
@@ -227,8 +234,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     if (best_cc >= 0) {
                         int idx = 0;
 #pragma unroll
-                        for (int q4 = 7; q4 >= 0; --q4) {            // lowest column that holds the maximum
-                            const float4 w = wrow[q4 ^ (row & 7)];
+                        for (int q4 = 3; q4 >= 0; --q4) {            // lowest column that holds the maximum
+                            const float4 w = wrow[q4];
                             if (w.w == best) idx = 4 * q4 + 3;
                             if (w.z == best) idx = 4 * q4 + 2;
                             if (w.y == best) idx = 4 * q4 + 1;

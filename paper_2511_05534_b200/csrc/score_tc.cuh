@@ -3,14 +3,14 @@
 //
 // The proxy attention needs every row's softmax normaliser before any column can be summed, so
 // the keys are streamed twice:
-//   pass 1  S = Q_group . K^T with the G*W proxy rows of a KV head as the 128 accumulator lanes
-//           and 256 keys per tile: each thread keeps the running maximum and exp-sum of its
-//           own row (no cross-thread traffic);
-//   pass 2  S^T = K . Q_group^T with 128 keys as the lanes and the proxy rows as columns: each
-//           thread owns one key, recomputes its logits, normalises them with the per-column
-//           constants of pass 1 and sums along its row, which is exactly the key's importance;
-//           the same probabilities, split by the modality of key and proxy token, give the
-//           cross-modal mass.
+//   pass 1  S = Q_group . K^T with the G*W proxy rows of a KV head as accumulator lanes (two
+//           halves of 128 rows per item) and 256 keys per tile: each thread keeps the running
+//           maximum and exp-sum of its own row (no cross-thread traffic);
+//   pass 2  S^T = K . Q_group^T with keys as the lanes (two halves of 128 keys per item) and the
+//           proxy rows as columns: each thread owns one key, recomputes its logits, normalises
+//           them with the per-column constants of pass 1 and sums along its row, which is
+//           exactly the key's importance; the same probabilities, split by the modality of key
+//           and proxy token, give the cross-modal mass.
 // Both passes run on tcgen05 with TMA-fed operands; logits never leave TMEM / registers.
 #pragma once
 #include "common.cuh"
@@ -23,34 +23,49 @@ struct ScoreTcArgs {
     float *negc;                 // [UH, GWpad] -(row max + log2 row sum); very negative for padding rows
     const uint8_t *modality;     // [U, L]
     float *importance;           // [UH, L]
-    float *cross_part;           // [U*Hq, n_rt * 4] partial cross-modal mass per key tile and epilogue warp
+    float *cross_part;           // [U*Hq, n_rt * 8] partial cross-modal mass per key tile and epilogue warp
     int *status;
     int Hq, Hkv, G, W, L, GW, GWpad;
-    int n_qt;                    // 128-row tiles over the G*W proxy rows
+    int n_qt;                    // 256-row tiles over the G*W proxy rows
     int n_chunk, tiles_per_chunk;   // pass 1: key chunks per row tile, 256-key tiles per chunk
-    int n_rt;                    // pass 2: 128-key tiles
+    int n_rt;                    // pass 2: 256-key tiles
     int a_heads, b_heads;        // query heads one A box (pass 1) / B box (pass 2) delivers
     int n_items1, n_items2;
     float scale_log2;
 };
 
+// max of 32 values with three-input maxima
+__device__ __forceinline__ float max32(const float (&v)[32]) {
+    float m12[12];
+#pragma unroll
+    for (int i = 0; i < 10; ++i) m12[i] = tc::max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
+    m12[10] = v[30]; m12[11] = v[31];
+    const float a0 = tc::max3(m12[0], m12[1], m12[2]), a1 = tc::max3(m12[3], m12[4], m12[5]);
+    const float a2 = tc::max3(m12[6], m12[7], m12[8]), a3 = tc::max3(m12[9], m12[10], m12[11]);
+    return fmaxf(tc::max3(a0, a1, a2), a3);
+}
+
 // ---------------------------------------------------------------------------------------------
-// Pass 1.  item = (unit*head, proxy row tile, key chunk).
+// Pass 1.  item = (unit*head, tile of 256 proxy rows, key chunk).
 __global__ void __launch_bounds__(tcs::kThreads, 1)
 score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                       const ScoreTcArgs A) {
-    extern __shared__ uint8_t smem_raw[];
-    const tcs::Ctx c = tcs::setup(smem_raw, &q_map, &k_map);
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const tcs::Ctx c = tcs::setup(smem_raw, &q_map, &k_map, A.status);
+    if (!c.ok) return;
     auto plan = [&](int item) {
         tcs::TilePlan p;
         const int kc = item % A.n_chunk, qt = (item / A.n_chunk) % A.n_qt, uh = item / (A.n_chunk * A.n_qt);
         const int u = uh / A.Hkv, h = uh % A.Hkv;
         const int key0 = kc * A.tiles_per_chunk * tcs::kCols;
         const int keys = min(A.L - key0, A.tiles_per_chunk * tcs::kCols);
-        p.a1 = 0; p.a2 = h * A.G + qt * (tcs::kRows / A.W); p.a3 = u;
+        p.a1 = 0; p.a2 = h * A.G + qt * (tcs::kItemRows / A.W); p.a3 = u;
+        p.h1 = 0; p.h2 = tcs::kRows / A.W;
+        p.n_halves = qt * tcs::kItemRows + tcs::kRows < A.GW ? 2 : 1;
         p.b1 = key0; p.b2 = h; p.b3 = u; p.step1 = tcs::kCols; p.step2 = 0;
         p.cols_total = keys > 0 ? keys : 0;
         p.n_tiles = (p.cols_total + tcs::kCols - 1) / tcs::kCols;
+        p.extra = nullptr;
         return p;
     };
     const uint32_t a_bytes = (uint32_t)A.a_heads * A.W * 256u;
@@ -59,59 +74,62 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
     } else if (c.warp == 1) {
         if (c.lane == 0) tcs::mma_issuer(c, A.n_items1, plan, A.status);
     } else {
-        const int row_in_tile = (c.warp & 3) * 32 + c.lane;
-        int tt = 0;
+        const int row_in_half = c.quarter * 32 + c.lane;
+        int k = 0;
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items1; item += gridDim.x) {
             const tcs::TilePlan p = plan(item);
+            if (p.empty() || c.group >= p.n_halves) continue;
             const int kc = item % A.n_chunk, qt = (item / A.n_chunk) % A.n_qt, uh = item / (A.n_chunk * A.n_qt);
-            const int r = qt * tcs::kRows + row_in_tile;
+            const int r = qt * tcs::kItemRows + c.group * tcs::kRows + row_in_half;
             const bool valid_row = r < A.GW;
-            const bool warp_has_rows = qt * tcs::kRows + (c.warp & 3) * 32 < A.GW;
+            const bool warp_has_rows = qt * tcs::kItemRows + c.group * tcs::kRows + c.quarter * 32 < A.GW;
             const int pa = A.L - A.W + (r % A.W);                    // last key this proxy row may see
             float m = kNegBig, l = 0.f;
-            for (int t = 0; ok && t < p.n_tiles; ++t, ++tt) {
-                ok = tcs::acc_wait(c, tt, A.status);
+            for (int t = 0; ok && t < p.n_tiles; ++t, ++k) {
+                ok = tcs::acc_wait(c, k, A.status);
                 if (!ok) break;
                 const int kb = p.b1 + t * tcs::kCols;
                 const int ncols = min(tcs::kCols, p.cols_total - t * tcs::kCols);
                 if (warp_has_rows) {
-                    for (int ch = 0; ch * 32 < ncols; ++ch) {
+                    tcs::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
                         const int k0 = kb + ch * 32;
-                        uint32_t acc[32];
-                        tc::tmem_ld32(tcs::acc_addr(c, tt, ch), acc);
-                        tc::tmem_ld_wait();
-                        float s[32];
+                        float mx;
+                        float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
                         if (k0 + 32 <= A.L - A.W + 1) {              // no key of this chunk is masked for any row
+                            float raw[32];
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) s[j] = __uint_as_float(acc[j]) * A.scale_log2;
+                            for (int j = 0; j < 32; ++j) raw[j] = __uint_as_float(acc[j]);
+                            mx = fmaxf(max32(raw) * A.scale_log2, m);
+                            const float neg = -mx;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                add0 += tc::ex2(fmaf(raw[j], A.scale_log2, neg));
+                                add1 += tc::ex2(fmaf(raw[j + 1], A.scale_log2, neg));
+                                add2 += tc::ex2(fmaf(raw[j + 2], A.scale_log2, neg));
+                                add3 += tc::ex2(fmaf(raw[j + 3], A.scale_log2, neg));
+                            }
                         } else {
+                            float s[32];
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
                                 s[j] = (k0 + j <= pa) ? __uint_as_float(acc[j]) * A.scale_log2 : kNegBig;
-                        }
-                        float m12[12];
+                            mx = fmaxf(max32(s), m);
 #pragma unroll
-                        for (int i = 0; i < 10; ++i) m12[i] = tc::max3(s[3 * i], s[3 * i + 1], s[3 * i + 2]);
-                        m12[10] = s[30]; m12[11] = s[31];
-                        const float a0 = tc::max3(m12[0], m12[1], m12[2]), a1 = tc::max3(m12[3], m12[4], m12[5]);
-                        const float a2 = tc::max3(m12[6], m12[7], m12[8]), a3 = tc::max3(m12[9], m12[10], m12[11]);
-                        const float mx = fmaxf(fmaxf(tc::max3(a0, a1, a2), a3), m);
-                        float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {            // masked entries sit ~1e30 below: exp2 gives 0
-                            add0 += tc::ex2(s[j] - mx);
-                            add1 += tc::ex2(s[j + 1] - mx);
-                            add2 += tc::ex2(s[j + 2] - mx);
-                            add3 += tc::ex2(s[j + 3] - mx);
+                            for (int j = 0; j < 32; j += 4) {        // masked entries sit ~1e30 below: exp2 gives 0
+                                add0 += tc::ex2(s[j] - mx);
+                                add1 += tc::ex2(s[j + 1] - mx);
+                                add2 += tc::ex2(s[j + 2] - mx);
+                                add3 += tc::ex2(s[j + 3] - mx);
+                            }
                         }
                         float add = (add0 + add1) + (add2 + add3);
                         if (mx < 0.5f * kNegBig) add = 0.f;          // nothing visible yet: exp2(0) terms are not real
                         l = l * tc::ex2(m - mx) + add;
                         m = mx;
-                    }
+                    });
                 }
-                tcs::acc_release(c, tt);
+                tcs::acc_release(c);
             }
             if (!ok) break;
             if (valid_row) A.row_part[((int64_t)uh * A.GW + r) * A.n_chunk + kc] = make_float2(m, l);
@@ -139,41 +157,45 @@ __global__ void score_combine_kernel(const float2 *row_part, int n_chunk, int GW
 }
 
 // ---------------------------------------------------------------------------------------------
-// Pass 2.  item = (unit*head, tile of 128 keys); the B stream is the head group's proxy rows.
+// Pass 2.  item = (unit*head, tile of 256 keys); the B stream is the head group's proxy rows.
 __global__ void __launch_bounds__(tcs::kThreads, 1)
 score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap q_map,
                        const ScoreTcArgs A) {
-    extern __shared__ uint8_t smem_raw[];
-    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &q_map);
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &q_map, A.status);
+    if (!c.ok) return;
     auto plan = [&](int item) {
         tcs::TilePlan p;
         const int kt = item % A.n_rt, uh = item / A.n_rt;
         const int u = uh / A.Hkv, h = uh % A.Hkv;
-        p.a1 = kt * tcs::kRows; p.a2 = h; p.a3 = u;
+        p.a1 = kt * tcs::kItemRows; p.a2 = h; p.a3 = u;
+        p.h1 = tcs::kRows; p.h2 = 0;
+        p.n_halves = p.a1 + tcs::kRows < A.L ? 2 : 1;
         p.b1 = 0; p.b2 = h * A.G; p.b3 = u; p.step1 = 0; p.step2 = tcs::kCols / A.W;
         p.cols_total = A.GW;
         p.n_tiles = (A.GW + tcs::kCols - 1) / tcs::kCols;
+        p.extra = A.negc + (int64_t)uh * A.GWpad;        // row constants of pass 1, 256 per B tile
         return p;
     };
     const uint32_t b_bytes = (uint32_t)A.b_heads * A.W * 256u;
     if (c.warp == 0) {
-        if (c.lane == 0) tcs::producer(c, &k_map, &q_map, A.n_items2, tcs::kAStage, b_bytes, plan, A.status);
+        if (c.lane == 0) tcs::producer(c, &k_map, &q_map, A.n_items2, tcs::kAHalf, b_bytes, plan, A.status);
     } else if (c.warp == 1) {
         if (c.lane == 0) tcs::mma_issuer(c, A.n_items2, plan, A.status);
     } else {
-        const int quarter = c.warp & 3, lane = c.lane;
-        float *negc_s = reinterpret_cast<float *>(c.epi_scratch()) + quarter * 1024;   // this warp's copy, <= 1024 rows
-        int tt = 0, cached_uh = -1, cached_u = -1;
+        const int lane = c.lane;
+        int k = 0, bt = 0, cached_u = -1;
         uint32_t wbits[4] = {0, 0, 0, 0};                            // modality of the proxy tokens, 32 per word
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items2; item += gridDim.x) {
             const tcs::TilePlan p = plan(item);
             const int kt = item % A.n_rt, uh = item / A.n_rt, u = uh / A.Hkv, h = uh % A.Hkv;
-            if (uh != cached_uh) {
-                __syncwarp();
-                for (int i = lane; i < A.GWpad; i += 32) negc_s[i] = A.negc[(int64_t)uh * A.GWpad + i];
-                __syncwarp();
-                cached_uh = uh;
+            float *cross_out = A.cross_part + ((int64_t)u * A.Hq + h * A.G) * (A.n_rt * 8) + kt * 8 + c.group * 4 + c.quarter;
+            if (c.group >= p.n_halves) {                             // no keys in this half: its masses are zero
+                if (lane == 0)
+                    for (int g = 0; g < A.G; ++g) cross_out[(int64_t)g * (A.n_rt * 8)] = 0.f;
+                bt += p.n_tiles;                                     // keep the B-tile count in step
+                continue;
             }
             if (u != cached_u) {
 #pragma unroll
@@ -184,40 +206,36 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                 }
                 cached_u = u;
             }
-            const int key = kt * tcs::kRows + quarter * 32 + lane;
-            const bool masked_tile = (kt + 1) * tcs::kRows > A.L - A.W + 1;   // some (key, proxy row) pair is masked
+            const int key0 = kt * tcs::kItemRows + c.group * tcs::kRows;
+            const int key = key0 + c.quarter * 32 + lane;
+            const bool masked_tile = key0 + tcs::kRows > A.L - A.W + 1;   // some (key, proxy row) pair is masked
             const bool my_vis = key < A.L && A.modality[(int64_t)u * A.L + key] != 0;
             const int first_proxy = A.L - A.W;
             float imp = 0.f, cg = 0.f;
             int cur_g = 0;
-            for (int t = 0; ok && t < p.n_tiles; ++t, ++tt) {
-                ok = tcs::acc_wait(c, tt, A.status);
-                if (!ok) break;
+            for (int t = 0; ok && t < p.n_tiles; ++t, ++k, ++bt) {
                 const int ncols = min(tcs::kCols, A.GW - t * tcs::kCols);
-                for (int ch = 0; ch * 32 < ncols; ++ch) {
+                const int n_chunks = (ncols + 31) >> 5;
+                ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
+                if (!ok) break;
+                const float4 *negc4 = c.extra(bt);
+                tcs::for_each_chunk(c, n_chunks, [&](int ch, uint32_t (&acc)[32]) {
                     const int col = t * tcs::kCols + ch * 32;        // proxy row index r = g_local * W + a
                     const int g_local = col / A.W, a0 = col % A.W;
                     if (g_local != cur_g) {                          // a head is complete: publish its mass
                         const float tot = warp_sum(cg);
-                        if (lane == 0)
-                            A.cross_part[((int64_t)u * A.Hq + h * A.G + cur_g) * (A.n_rt * 4) + kt * 4 + quarter] = tot;
+                        if (lane == 0) cross_out[(int64_t)cur_g * (A.n_rt * 8)] = tot;
                         cg = 0.f;
                         cur_g = g_local;
                     }
-                    uint32_t acc[32];
-                    tc::tmem_ld32(tcs::acc_addr(c, tt, ch), acc);
-                    const float4 *np = reinterpret_cast<const float4 *>(negc_s + col);
-                    float4 n4[8];
-#pragma unroll
-                    for (int q4 = 0; q4 < 8; ++q4) n4[q4] = np[q4];
-                    tc::tmem_ld_wait();
                     float pr[32];
 #pragma unroll
                     for (int q4 = 0; q4 < 8; ++q4) {
-                        pr[4 * q4 + 0] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 0]), A.scale_log2, n4[q4].x));
-                        pr[4 * q4 + 1] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 1]), A.scale_log2, n4[q4].y));
-                        pr[4 * q4 + 2] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 2]), A.scale_log2, n4[q4].z));
-                        pr[4 * q4 + 3] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 3]), A.scale_log2, n4[q4].w));
+                        const float4 n4 = negc4[ch * 8 + q4];
+                        pr[4 * q4 + 0] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 0]), A.scale_log2, n4.x));
+                        pr[4 * q4 + 1] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 1]), A.scale_log2, n4.y));
+                        pr[4 * q4 + 2] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 2]), A.scale_log2, n4.z));
+                        pr[4 * q4 + 3] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 3]), A.scale_log2, n4.w));
                     }
                     if (masked_tile) {                               // causal mask inside the window, and keys >= L
 #pragma unroll
@@ -238,14 +256,13 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                         for (int j = 0; j < 32; ++j) x += ((other >> j) & 1u) ? pr[j] : 0.f;
                         cg += x;
                     }
-                }
-                tcs::acc_release(c, tt);
+                });
+                tcs::acc_release(c);
             }
             if (!ok) break;
             {
                 const float tot = warp_sum(cg);
-                if (lane == 0)
-                    A.cross_part[((int64_t)u * A.Hq + h * A.G + cur_g) * (A.n_rt * 4) + kt * 4 + quarter] = tot;
+                if (lane == 0) cross_out[(int64_t)cur_g * (A.n_rt * 8)] = tot;
             }
             if (key < A.L) A.importance[(int64_t)uh * A.L + key] = imp / (float)A.G;     // group mean
         }
