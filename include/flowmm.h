@@ -164,9 +164,9 @@ flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v,
  * flowmm_merge (same kernels, same fixed accumulation order, so the outputs are bit-identical).
  *
  * Limits and rules:
- *   - The scratch a problem needs is about 8 E + 12 (B + 1) bytes per (unit, KV head) plus
- *     (2 E / 64 + 2) * (8 head_dim + 16) bytes per (unit, KV head) of partial sums; if that
- *     exceeds the array the call returns FLOWMM_ERR_WORKSPACE and launches nothing.
+ *   - The scratch a problem needs is about 16 E + 28 (B + 1) + E / 4 bytes per (unit, KV head)
+ *     plus (2 E / 64 + 2) * (8 head_dim + 16) bytes per (unit, KV head) of partial sums; if
+ *     that exceeds the array the call returns FLOWMM_ERR_WORKSPACE and launches nothing.
  *   - The first call on a device looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array and it keeps the previous call's contents;

@@ -17,6 +17,10 @@ template <> struct Elem<float> {
         const float4 v = *reinterpret_cast<const float4 *>(p);
         out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
     }
+    __device__ static void unpack(const uint4 &v, float (&out)[4]) {
+        out[0] = __uint_as_float(v.x); out[1] = __uint_as_float(v.y);
+        out[2] = __uint_as_float(v.z); out[3] = __uint_as_float(v.w);
+    }
     __device__ static void store16(float *p, const float (&in)[4]) {
         *reinterpret_cast<float4 *>(p) = make_float4(in[0], in[1], in[2], in[3]);
     }
@@ -32,6 +36,14 @@ template <> struct Elem<__nv_bfloat16> {
             out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
     }
+    __device__ static void unpack(const uint4 &v, float (&out)[8]) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            out[2 * i] = __uint_as_float(w[i] << 16);
+            out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
     __device__ static void store16(__nv_bfloat16 *p, const float (&in)[8]) {
         uint32_t w[4];
 #pragma unroll
@@ -42,6 +54,11 @@ template <> struct Elem<__nv_bfloat16> {
         *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 };
+
+// 16 bytes of a row as they are in memory; Elem<T>::unpack turns them into floats
+template <typename T> __device__ __forceinline__ uint4 load_raw16(const T *p) {
+    return *reinterpret_cast<const uint4 *>(p);
+}
 
 // ---- warp helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float warp_sum(float v) {

@@ -55,7 +55,7 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // Where everything lives inside the caller's workspace.  One layout serves every entry point.
 struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
-    size_t row_part, cross_part, rn, sort_a, sort_b, off, piece_off, part_off, partial;
+    size_t row_part, cross_part, rn, sort_a, sort_b, mem_tok, mem_w, piece_desc, off, piece_off, part_off, partial;
     size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod, negc;
     int tc_n_qt, tc_n_chunk, tc_tiles_per_chunk, gw_pad;
     size_t total;
@@ -72,6 +72,25 @@ int chunks_for(int L, int other_ctas, int &chunk) {
     return (L + chunk - 1) / chunk;
 }
 
+// The part of the workspace that the merge step uses (CSR of the match, piece table, partial sums).
+template <class Take>
+void layout_merge(Layout &y, const flowmm_params &p, Take take) {
+    const size_t UH = (size_t)p.n_units * p.n_kv_heads, B = p.n_keep, E = (size_t)p.seq_len - B, D = p.head_dim;
+    y.max_pieces = (int)(B + E / kPiece + 1);
+    y.max_parts = (int)(2 * (E / kPiece) + 2);
+    y.csr_passes = 1;
+    while (y.csr_passes < 4 && (B >> (8 * y.csr_passes)) != 0) ++y.csr_passes;
+    y.sort_a = take(UH * E * 4);
+    y.sort_b = take(UH * E * 4);
+    y.mem_tok = take(UH * E * 4);
+    y.mem_w = take(UH * E * 4);
+    y.piece_desc = take(UH * (size_t)y.max_pieces * 16);
+    y.off = take(UH * (B + 1) * 4);
+    y.piece_off = take(UH * (B + 1) * 4);
+    y.part_off = take(UH * (B + 1) * 4);
+    y.partial = take(UH * (size_t)y.max_parts * (2 * D + 4) * 4);
+}
+
 Layout make_layout(const flowmm_params &p) {
     Layout y;
     const size_t U = p.n_units, Hq = p.n_q_heads, Hkv = p.n_kv_heads, L = p.seq_len, W = p.window;
@@ -79,10 +98,6 @@ Layout make_layout(const flowmm_params &p) {
     const int row_tiles = (int)((G * W + kTile - 1) / kTile);
     y.n_chunk1 = chunks_for((int)L, (int)(U * Hkv) * row_tiles, y.chunk1);
     y.n_chunk2 = chunks_for((int)L, (int)(U * Hkv), y.chunk2);
-    y.max_pieces = (int)(B + E / kPiece + 1);
-    y.max_parts = (int)(2 * (E / kPiece) + 2);
-    y.csr_passes = 1;
-    while (y.csr_passes < 4 && (B >> (8 * y.csr_passes)) != 0) ++y.csr_passes;
     size_t o = 0;
     auto take = [&](size_t bytes) { const size_t at = o; o += align256(bytes); return at; };
     y.status = take(256);
@@ -118,12 +133,7 @@ Layout make_layout(const flowmm_params &p) {
     y.cross_part = take(U * Hq * max_chunk2 * 4);
     y.negc = take(U * Hkv * (size_t)y.gw_pad * 4);
     y.rn = take(U * Hkv * L * 4);
-    y.sort_a = take(U * Hkv * E * 4);
-    y.sort_b = take(U * Hkv * E * 4);
-    y.off = take(U * Hkv * (B + 1) * 4);
-    y.piece_off = take(U * Hkv * (B + 1) * 4);
-    y.part_off = take(U * Hkv * (B + 1) * 4);
-    y.partial = take(U * Hkv * (size_t)y.max_parts * (2 * D + 4) * 4);
+    layout_merge(y, p, take);
     y.c_tot = (int)((B + 31) / 32 * 32 + 32);
     y.cand_k = take(U * Hkv * (size_t)y.c_tot * 128 * 2);
     y.cand_scale = take(U * Hkv * (size_t)y.c_tot * 4 + 1024);   // + one tile of slack: whole 256-column slices are copied
@@ -277,7 +287,8 @@ flowmm_status run_layer_flow(const flowmm_params &p, const float *cross_mass, fl
 
 flowmm_status run_select(const flowmm_params &p, const float *importance, int32_t *retained, int32_t *evicted,
                          cudaStream_t st) {
-    select_topb_kernel<<<p.n_units * p.n_kv_heads, kSelectThreads, 0, st>>>(importance, p.seq_len, p.n_keep, p.window,
+    const int threads = p.seq_len <= 2048 ? 256 : p.seq_len <= 8192 ? 512 : kSelectThreads;
+    select_topb_kernel<<<p.n_units * p.n_kv_heads, threads, 0, st>>>(importance, p.seq_len, p.n_keep, p.window,
                                                                            p.keep_window, retained, evicted);
     FLOWMM_LAUNCHED("select_topb");
     return FLOWMM_OK;
@@ -289,7 +300,7 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
                            const int32_t *strategy, int32_t *match, float *match_sim, void *ws, cudaStream_t st) {
     const int UH = p.n_units * p.n_kv_heads, E = p.seq_len - p.n_keep;
     MatchPrepArgs g;
-    g.k = k; g.importance = importance; g.rn = at<float>(ws, y.rn); g.modality = mod;
+    g.k = k; g.importance = importance; g.modality = mod;
     g.retained = retained; g.evicted = evicted;
     g.cand_k = at<__nv_bfloat16>(ws, y.cand_k); g.cand_scale = at<float>(ws, y.cand_scale);
     g.cand_slot = at<int>(ws, y.cand_slot); g.cand_count = at<int>(ws, y.cand_count);
@@ -310,7 +321,7 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
         return FLOWMM_ERR_CUDA;
     MatchTcArgs a;
     a.cand_count = g.cand_count; a.cand_slot = g.cand_slot; a.rank = g.rank; a.strategy = strategy;
-    a.cand_scale = g.cand_scale; a.rn = g.rn; a.modality = mod; a.tile_mod = g.tile_mod;
+    a.cand_scale = g.cand_scale; a.modality = mod; a.tile_mod = g.tile_mod;
     a.match = match; a.match_sim = match_sim; a.status = at<int>(ws, y.status);
     a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.E = E; a.Ctot = y.c_tot; a.n_rt = y.n_rt; a.n_items = UH * y.n_rt;
     if (cudaFuncSetAttribute(match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tcs::kSmemBytes) !=
@@ -327,6 +338,7 @@ flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, 
                         int32_t *match, float *match_sim, void *ws, cudaStream_t st) {
     const int E = p.seq_len - p.n_keep;
     if (E == 0) return FLOWMM_OK;
+    if (use_tc(p)) return run_match_tc(p, y, k, importance, mod, retained, evicted, strategy, match, match_sim, ws, st);
     float *rn = at<float>(ws, y.rn);
     const int64_t rows = (int64_t)p.n_units * p.n_kv_heads * p.seq_len;
     const int lanes = p.head_dim / (p.dtype == FLOWMM_BF16 ? 8 : 4);
@@ -339,7 +351,6 @@ flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, 
         inv_norm_kernel<float><<<blocks, 256, 0, st>>>(k, rows, p.n_kv_heads, p.seq_len, p.head_dim, p.k_stride[0],
                                                        p.k_stride[1], p.k_stride[2], rn);
     FLOWMM_LAUNCHED("inv_norm");
-    if (use_tc(p)) return run_match_tc(p, y, k, importance, mod, retained, evicted, strategy, match, match_sim, ws, st);
     MatchArgs a;
     a.k = k; a.importance = importance; a.modality = mod; a.retained = retained; a.evicted = evicted;
     a.strategy = strategy; a.rn = rn; a.match = match; a.match_sim = match_sim;
@@ -358,32 +369,38 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
                         void *k_out, void *v_out, void *ws, cudaStream_t st) {
     const int E = p.seq_len - p.n_keep, UH = p.n_units * p.n_kv_heads;
     MergeArgs m;
-    m.k = k; m.v = v; m.k_out = k_out; m.v_out = v_out; m.retained = retained; m.evicted = evicted;
-    m.match_sim = match_sim;
-    m.sorted = nullptr; m.off = nullptr; m.piece_off = nullptr; m.part_off = nullptr;
+    m.k = k; m.v = v; m.k_out = k_out; m.v_out = v_out; m.retained = retained;
+    m.mem_tok = nullptr; m.mem_w = nullptr; m.piece_desc = nullptr; m.piece_off = nullptr; m.part_off = nullptr;
     m.partial = at<float>(ws, y.partial);
     m.Hkv = p.n_kv_heads; m.D = p.head_dim; m.L = p.seq_len; m.B = p.n_keep; m.E = E;
-    m.max_pieces = E == 0 ? p.n_keep : y.max_pieces; m.max_parts = y.max_parts; m.merge_mode = p.merge_mode;
+    m.max_pieces = E == 0 ? p.n_keep : y.max_pieces; m.max_parts = y.max_parts;
     for (int i = 0; i < 3; ++i) {
         m.ks[i] = p.k_stride[i]; m.vs[i] = p.v_stride[i]; m.kos[i] = p.ko_stride[i]; m.vos[i] = p.vo_stride[i];
     }
     if (E > 0) {
         CsrArgs c;
-        c.match = match; c.sort_a = at<int>(ws, y.sort_a); c.sort_b = at<int>(ws, y.sort_b);
+        c.match = match; c.evicted = evicted; c.match_sim = match_sim;
+        c.sort_a = at<int>(ws, y.sort_a); c.sort_b = at<int>(ws, y.sort_b);
+        c.mem_tok = at<int>(ws, y.mem_tok); c.mem_w = at<float>(ws, y.mem_w);
         c.off = at<int>(ws, y.off); c.piece_off = at<int>(ws, y.piece_off); c.part_off = at<int>(ws, y.part_off);
-        c.B = p.n_keep; c.E = E; c.n_pass = y.csr_passes;
-        build_csr_kernel<<<UH, kCsrThreads, 0, st>>>(c);
+        c.piece_desc = at<int4>(ws, y.piece_desc);
+        c.B = p.n_keep; c.E = E; c.n_pass = y.csr_passes; c.max_pieces = y.max_pieces; c.merge_mode = p.merge_mode;
+        if (E <= 4096) build_csr_kernel<8><<<UH, 256, 0, st>>>(c);
+        else build_csr_kernel<32><<<UH, 1024, 0, st>>>(c);
         FLOWMM_LAUNCHED("build_csr");
-        m.sorted = ((y.csr_passes - 1) & 1) ? c.sort_b : c.sort_a;
-        m.off = c.off; m.piece_off = c.piece_off; m.part_off = c.part_off;
+        m.mem_tok = c.mem_tok; m.mem_w = c.mem_w; m.piece_desc = c.piece_desc;
+        m.piece_off = c.piece_off; m.part_off = c.part_off;
     }
-    const dim3 gp((m.max_pieces + 7) / 8, UH), gf((p.n_keep + 7) / 8, UH);
+    const int64_t total_pieces = (int64_t)UH * m.max_pieces;
+    const int64_t want_blocks = (total_pieces + 7) / 8;
+    const int gp = (int)(want_blocks < 2 * tc::sm_count() ? want_blocks : 2 * tc::sm_count());   // persistent warps
+    const dim3 gf((p.n_keep + 7) / 8, UH);
     if (p.dtype == FLOWMM_BF16) {
-        merge_pieces_kernel<__nv_bfloat16><<<gp, 256, 0, st>>>(m);
+        merge_pieces_kernel<__nv_bfloat16><<<gp, 256, 0, st>>>(m, UH);
         FLOWMM_LAUNCHED("merge_pieces");
         if (E > kPiece) { merge_finish_kernel<__nv_bfloat16><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCHED("merge_finish"); }
     } else {
-        merge_pieces_kernel<float><<<gp, 256, 0, st>>>(m);
+        merge_pieces_kernel<float><<<gp, 256, 0, st>>>(m, UH);
         FLOWMM_LAUNCHED("merge_pieces");
         if (E > kPiece) { merge_finish_kernel<float><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCHED("merge_finish"); }
     }
@@ -592,19 +609,8 @@ flowmm_status merge_static_base(void **base) {
 // The part of the workspace layout that the merge step touches, packed from offset 0.
 Layout make_merge_layout(const flowmm_params &p) {
     Layout y = {};
-    const size_t UH = (size_t)p.n_units * p.n_kv_heads, B = p.n_keep, E = (size_t)p.seq_len - B, D = p.head_dim;
-    y.max_pieces = (int)(B + E / kPiece + 1);
-    y.max_parts = (int)(2 * (E / kPiece) + 2);
-    y.csr_passes = 1;
-    while (y.csr_passes < 4 && (B >> (8 * y.csr_passes)) != 0) ++y.csr_passes;
     size_t o = 0;
-    auto take = [&](size_t bytes) { const size_t at = o; o += align256(bytes); return at; };
-    y.sort_a = take(UH * E * 4);
-    y.sort_b = take(UH * E * 4);
-    y.off = take(UH * (B + 1) * 4);
-    y.piece_off = take(UH * (B + 1) * 4);
-    y.part_off = take(UH * (B + 1) * 4);
-    y.partial = take(UH * (size_t)y.max_parts * (2 * D + 4) * 4);
+    layout_merge(y, p, [&](size_t bytes) { const size_t at = o; o += align256(bytes); return at; });
     y.total = o;
     return y;
 }

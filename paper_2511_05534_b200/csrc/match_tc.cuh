@@ -21,7 +21,7 @@ constexpr int kMtCols = tcs::kCols;          // candidates per column tile
 
 struct MatchPrepArgs {
     const void *k;
-    const float *importance, *rn;
+    const float *importance;
     const uint8_t *modality;
     const int *retained, *evicted;
     __nv_bfloat16 *cand_k;       // [UH, Ctot, 128]
@@ -43,7 +43,6 @@ __global__ void __launch_bounds__(256) match_prepare_kernel(const MatchPrepArgs 
     const int *ret = A.retained + (int64_t)uh * A.B;
     const int *evi = A.evicted + (int64_t)uh * A.E;
     const float *imp = A.importance + (int64_t)uh * A.L;
-    const float *rn = A.rn + (int64_t)uh * A.L;
     const uint8_t *mod = A.modality + (int64_t)u * A.L;
     int *rank = A.rank + (int64_t)uh * A.L;
     int *slot_out = A.cand_slot + (int64_t)uh * A.Ctot;
@@ -84,28 +83,36 @@ __global__ void __launch_bounds__(256) match_prepare_kernel(const MatchPrepArgs 
         int tot_t, tot_v;
         const int pt = seen_t + block_exclusive_scan(ft, scratch, tot_t);
         const int pv = seen_v + block_exclusive_scan(fv, scratch, tot_v);
-        if (ft) { slot_out[pt] = s; scale_out[pt] = rn[r]; }
-        if (fv) { slot_out[t0 + pv] = s; scale_out[t0 + pv] = rn[r]; }
+        if (ft) slot_out[pt] = s;
+        if (fv) slot_out[t0 + pv] = s;
         seen_t += tot_t;
         seen_v += tot_v;
     }
     if (tid == 0) { A.cand_count[2 * uh] = seen_t; A.cand_count[2 * uh + 1] = seen_v; }
     __syncthreads();
-    // copy the candidate key rows (256 bytes each): 16 lanes per row
+    // copy the candidate key rows (256 bytes each), 16 lanes per row, and take each row's reciprocal
+    // norm on the way (0 for a zero row: its similarity to anything is 0)
     const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(A.k) + u * A.ks[0] + h * A.ks[1];
     uint4 *dst = reinterpret_cast<uint4 *>(A.cand_k + (int64_t)uh * A.Ctot * 128);
     const int sub = tid & 15;
-    for (int pos = tid >> 4; pos < A.Ctot; pos += blockDim.x >> 4) {
+    for (int pos = tid >> 4; pos < A.Ctot; pos += blockDim.x >> 4) {        // Ctot is a multiple of 32: uniform trip count
         const int s = slot_out[pos];
         uint4 val = make_uint4(0, 0, 0, 0);
         if (s >= 0) val = *reinterpret_cast<const uint4 *>(kb + (int64_t)ret[s] * A.ks[2] + sub * 8);
         dst[(int64_t)pos * 16 + sub] = val;
+        float x[8], ssq = 0.f;
+        Elem<__nv_bfloat16>::unpack(val, x);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xFFFFFFFFu, ssq, o);
+        if (sub == 0 && s >= 0) scale_out[pos] = ssq > 0.f ? rsqrtf(ssq) : 0.f;
     }
 }
 
 struct MatchTcArgs {
     const int *cand_count, *cand_slot, *rank, *strategy;
-    const float *cand_scale, *rn;
+    const float *cand_scale;
     const uint8_t *modality, *tile_mod;
     int *match;
     float *match_sim;
@@ -151,7 +158,7 @@ __global__ void __launch_bounds__(tcs::kThreads, 1)
 match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap cand_map,
                 const MatchTcArgs A) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &cand_map, A.status);
+    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &cand_map, A.status, 4);
     if (!c.ok) return;
     auto plan = [&](int item) { return match_plan(A, item).tp; };
     if (c.warp == 0) {
@@ -161,7 +168,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
         float4 *wrow = reinterpret_cast<float4 *>(c.epi_scratch()) + row * 4;   // 16 floats per row
-        int k = 0, bt = 0;
+        int k = 0, bt = 0, n_mine = 0;
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
             const MatchItem p = match_plan(A, item);
@@ -175,9 +182,27 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             const bool row_masked = p.intra && p.mixed;
             float best = -INFINITY;
             int best_cc = -1;
+            float ssq = 0.f;                                         // squared norm of this row's key
             if (!active) {
                 if (!p.tp.empty()) bt += p.tp.n_tiles;               // keep the B-tile count in step
             } else {
+                // the token's key row sits in this half's A stage (128-byte rows, 16-byte units XOR-swizzled by
+                // the row index): read it once for the norm while the first MMAs run, then hand the stage back
+                ok = tcs::a_wait(c, n_mine++, A.status);
+                if (!ok) break;
+                const uint8_t *a_half = c.gen + tcs::kSmemA + c.group * tcs::kAHalf + row * 128;
+#pragma unroll
+                for (int kh = 0; kh < 2; ++kh) {
+#pragma unroll
+                    for (int un = 0; un < 8; ++un) {
+                        const uint4 raw = *reinterpret_cast<const uint4 *>(a_half + kh * (tcs::kAHalf / 2) + ((un ^ (row & 7)) << 4));
+                        float x[8];
+                        Elem<__nv_bfloat16>::unpack(raw, x);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
+                    }
+                }
+                tcs::a_release(c);
                 for (int t = 0; ok && t < p.tp.n_tiles; ++t, ++k, ++bt) {
                     const int col0 = p.lo + t * kMtCols;
                     const int ncols = min(kMtCols, p.hi - col0);
@@ -242,7 +267,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                             if (w.x == best) idx = 4 * q4;
                         }
                         slot = A.cand_slot[(int64_t)p.uh * A.Ctot + best_cc + idx];
-                        sim = best * A.rn[(int64_t)p.uh * A.L + token];
+                        sim = ssq > 0.f ? best * rsqrtf(ssq) : 0.f;
                     }
                     A.match[(int64_t)p.uh * A.E + j] = slot;
                     A.match_sim[(int64_t)p.uh * A.E + j] = sim;

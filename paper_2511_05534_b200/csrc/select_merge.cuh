@@ -16,14 +16,14 @@ __device__ __forceinline__ uint32_t select_key(float v, bool forced) {
 
 // Section 3.3.1 pivot selection: a radix select finds the B-th largest key, then one ordered
 // sweep writes the pivot positions and the non-pivot positions, both ascending.  Ties at the
-// threshold go to the lower positions.  grid = U*Hkv, block = 1024.
+// threshold go to the lower positions.  grid = U*Hkv, block = any multiple of 32 up to 1024.
 __global__ void __launch_bounds__(kSelectThreads)
 select_topb_kernel(const float *importance, int L, int B, int W, int keep_window, int *retained, int *evicted) {
     __shared__ int hist[256];
     __shared__ int scratch[33];
     __shared__ uint32_t s_prefix;
     __shared__ int s_need;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, nthreads = blockDim.x, lane = tid & 31;
     const float *imp = importance + (int64_t)blockIdx.x * L;
     int *ret = retained + (int64_t)blockIdx.x * B;
     int *evi = evicted + (int64_t)blockIdx.x * (L - B);
@@ -33,31 +33,42 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
     uint32_t prefix = 0, mask = 0;
     int need = B;                                    // how many keys to take among those matching prefix
     for (int shift = 24; shift >= 0; shift -= 8) {
-        if (tid < 256) hist[tid] = 0;
+        for (int i = tid; i < 256; i += nthreads) hist[i] = 0;
         __syncthreads();
-        for (int i = tid; i < L; i += kSelectThreads) {
+        for (int i = tid; i < L; i += nthreads) {
             const uint32_t key = select_key(imp[i], i >= first_forced);
             if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
         }
         __syncthreads();
-        if (tid == 0) {
-            int acc = 0, d = 255;
-            for (; d > 0; --d) {                     // walk down from the largest digit
-                if (acc + hist[d] >= need) break;
-                acc += hist[d];
+        if (tid < 32) {                              // walk down from the largest digit, 8 digits per lane
+            int local[8], lsum = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { local[e] = hist[255 - (lane * 8 + e)]; lsum += local[e]; }
+            int incl = lsum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += t;
             }
-            s_prefix = prefix | ((uint32_t)d << shift);
-            s_need = need - acc;
+            int acc = incl - lsum;                   // keys with a larger digit than this lane's first
+            if (acc < need && need <= incl) {        // the B-th largest key has one of this lane's digits
+                int e = 0;
+                for (; e < 7; ++e) {
+                    if (acc + local[e] >= need) break;
+                    acc += local[e];
+                }
+                s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + e)) << shift);
+                s_need = need - acc;
+            }
         }
         __syncthreads();
         prefix = s_prefix;
         need = s_need;
         mask |= 0xFFu << shift;
-        __syncthreads();
     }
     // keys > prefix are all kept; of the keys == prefix the first `need` (by position) are kept
     int eq_seen = 0, kept_seen = 0;
-    for (int base = 0; base < L; base += kSelectThreads) {
+    for (int base = 0; base < L; base += nthreads) {
         const int i = base + tid;
         uint32_t key = 0;
         bool valid = i < L;
@@ -80,39 +91,47 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
 // ---------------------------------------------------------------------------------------------
 // Merge stage.  The match array maps non-pivot j to a slot (or -1).  The members of every slot
 // are needed in a fixed order, so the non-pivot positions j are sorted by slot with a stable
-// LSD radix sort (ascending j inside a slot); slot s then owns sorted[off[s] .. off[s+1]).
-// Long member lists are cut into pieces of kPiece so that many warps share a popular pivot.
+// LSD radix sort (ascending j inside a slot); slot s then owns entries off[s] .. off[s+1] of the
+// sorted order, for which the kernel writes the member's token position and Eq. 5 weight.
+// Long member lists are cut into pieces of kPiece so that many warps share a popular pivot; one
+// descriptor per piece tells its warp what to do without any search.
 // ---------------------------------------------------------------------------------------------
-constexpr int kCsrThreads = 1024;
 constexpr int kPiece = 64;
 
 struct CsrArgs {
     const int *match;        // [UH, E]
+    const int *evicted;      // [UH, E]
+    const float *match_sim;  // [UH, E]
     int *sort_a, *sort_b;    // [UH, E] ping-pong buffers of non-pivot positions
+    int *mem_tok;            // [UH, E] token position of the i-th member in slot order
+    float *mem_w;            // [UH, E] its merge weight
     int *off;                // [UH, B+1] first member of each slot in the sorted order
     int *piece_off;          // [UH, B+1] first piece of each slot
     int *part_off;           // [UH, B+1] first partial-sum record of each slot (multi-piece slots only)
-    int B, E, n_pass;
+    int4 *piece_desc;        // [UH, max_pieces] (slot, first member, members, partial record or -1)
+    int B, E, n_pass, max_pieces, merge_mode;
 };
 
 __device__ __forceinline__ int csr_key(int m, int B) { return m < 0 ? B : m; }   // dropped tokens sort last
 
-// grid = U*Hkv, block = 1024 (32 warps; warp w owns a contiguous range of the input).
-__global__ void __launch_bounds__(kCsrThreads) build_csr_kernel(const CsrArgs A) {
-    __shared__ int counters[32][257];               // [warp][digit], padded
+// grid = U*Hkv, block = 32 * NW threads (warp w owns a contiguous range of the input).
+template <int NW>
+__global__ void __launch_bounds__(32 * NW) build_csr_kernel(const CsrArgs A) {
+    constexpr int kThreads = 32 * NW;
+    __shared__ int counters[NW][257];               // [warp][digit], padded
     __shared__ int scratch[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int uh = blockIdx.x;
     const int *match = A.match + (int64_t)uh * A.E;
     int *bufs[2] = {A.sort_a + (int64_t)uh * A.E, A.sort_b + (int64_t)uh * A.E};
-    const int per_warp = ((A.E + 31) / 32 + 31) / 32 * 32;     // multiple of 32
+    const int per_warp = ((A.E + NW - 1) / NW + 31) / 32 * 32;     // multiple of 32
     const int lo = warp * per_warp, hi = min(A.E, lo + per_warp);
 
     for (int pass = 0; pass < A.n_pass; ++pass) {
         const int shift = 8 * pass;
         const int *src = pass == 0 ? nullptr : bufs[(pass - 1) & 1];
         int *dst = bufs[pass & 1];
-        for (int i = tid; i < 32 * 257; i += kCsrThreads) (&counters[0][0])[i] = 0;
+        for (int i = tid; i < NW * 257; i += kThreads) (&counters[0][0])[i] = 0;
         __syncthreads();
         // count digits, warp-private counters
         for (int t = lo; t < lo + per_warp && t < ((hi + 31) / 32) * 32; t += 32) {
@@ -129,8 +148,8 @@ __global__ void __launch_bounds__(kCsrThreads) build_csr_kernel(const CsrArgs A)
         int vals[8], sum = 0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const int idx = tid * 8 + e;            // idx = digit * 32 + warp
-            vals[e] = counters[idx & 31][idx >> 5];
+            const int idx = tid * 8 + e;            // idx = digit * NW + warp
+            vals[e] = counters[idx % NW][idx / NW];
             sum += vals[e];
         }
         int total;
@@ -138,7 +157,7 @@ __global__ void __launch_bounds__(kCsrThreads) build_csr_kernel(const CsrArgs A)
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const int idx = tid * 8 + e;
-            counters[idx & 31][idx >> 5] = run;
+            counters[idx % NW][idx / NW] = run;
             run += vals[e];
         }
         __syncthreads();
@@ -162,8 +181,20 @@ __global__ void __launch_bounds__(kCsrThreads) build_csr_kernel(const CsrArgs A)
     int *off = A.off + (int64_t)uh * (A.B + 1);
     int *piece_off = A.piece_off + (int64_t)uh * (A.B + 1);
     int *part_off = A.part_off + (int64_t)uh * (A.B + 1);
+    // token position and weight of every member, in slot order
+    {
+        const int *evi = A.evicted + (int64_t)uh * A.E;
+        const float *sim = A.match_sim + (int64_t)uh * A.E;
+        int *mem_tok = A.mem_tok + (int64_t)uh * A.E;
+        float *mem_w = A.mem_w + (int64_t)uh * A.E;
+        for (int i = tid; i < A.E; i += kThreads) {
+            const int j = sorted[i];
+            mem_tok[i] = evi[j];
+            mem_w[i] = A.merge_mode == 1 ? 1.f : __expf(sim[j] - 1.f);
+        }
+    }
     // off[s] = number of sorted entries with key < s (binary search on the sorted order)
-    for (int s = tid; s <= A.B; s += kCsrThreads) {
+    for (int s = tid; s <= A.B; s += kThreads) {
         int a = 0, b = A.E;
         while (a < b) {
             const int mid = (a + b) >> 1;
@@ -173,12 +204,13 @@ __global__ void __launch_bounds__(kCsrThreads) build_csr_kernel(const CsrArgs A)
     }
     __syncthreads();
     // pieces per slot and partial records per slot, exclusive scans over the slots
+    int4 *desc = A.piece_desc + (int64_t)uh * A.max_pieces;
     int piece_seen = 0, part_seen = 0;
-    for (int base = 0; base <= A.B; base += kCsrThreads) {
+    for (int base = 0; base <= A.B; base += kThreads) {
         const int s = base + tid;
-        int np = 0, npart = 0;
+        int n = 0, np = 0, npart = 0;
         if (s < A.B) {
-            const int n = off[s + 1] - off[s];
+            n = off[s + 1] - off[s];
             np = n > kPiece ? (n + kPiece - 1) / kPiece : 1;
             npart = np > 1 ? np : 0;
         }
@@ -186,116 +218,137 @@ __global__ void __launch_bounds__(kCsrThreads) build_csr_kernel(const CsrArgs A)
         const int pp = piece_seen + block_exclusive_scan(np, scratch, tot_p);
         const int qq = part_seen + block_exclusive_scan(npart, scratch, tot_q);
         if (s <= A.B) { piece_off[s] = pp; part_off[s] = qq; }
+        for (int q = 0; q < np; ++q)
+            desc[pp + q] = make_int4(s, off[s] + q * kPiece, min(kPiece, n - q * kPiece), np > 1 ? qq + q : -1);
         piece_seen += tot_p;
         part_seen += tot_q;
     }
+    for (int i = piece_seen + tid; i < A.max_pieces; i += kThreads) desc[i] = make_int4(0, 0, -1, -1);   // unused entries
 }
 
 struct MergeArgs {
     const void *k, *v;
     void *k_out, *v_out;
-    const int *retained, *evicted;    // [UH, B], [UH, E]
-    const float *match_sim;           // [UH, E]
-    const int *sorted, *off, *piece_off, *part_off;   // CSR arrays; all nullptr when E == 0
+    const int *retained;              // [UH, B]
+    const int *mem_tok;               // [UH, E] member token positions in slot order; nullptr when E == 0
+    const float *mem_w;               // [UH, E] member weights
+    const int4 *piece_desc;           // [UH, max_pieces]
+    const int *piece_off, *part_off;  // [UH, B+1]
     float *partial;                   // [UH, max_parts, 2*D + 4] fp32 partial sums
-    int Hkv, D, L, B, E, max_pieces, max_parts, merge_mode;
+    int Hkv, D, L, B, E, max_pieces, max_parts;
     int64_t ks[3], vs[3], kos[3], vos[3];
 };
 
-// One warp per piece of a slot.  A 16-byte vector of a K row or V row per lane: with D*sizeof(T)
-// = 256 bytes lanes 0-15 carry the K row and lanes 16-31 the V row.  A single-piece slot is
-// finished here (pivot row with weight 1, Eq. 5 weights, normalise, round once); a piece of a
-// multi-piece slot stores its fp32 partial sums for merge_finish_kernel.
-// grid = (ceil(max_pieces / warps per block), U*Hkv).
+constexpr int kMergeBatch = 8;        // member rows a warp keeps in flight
+
+// One warp per piece of a slot, persistent: a warp walks the flat piece table with a stride and
+// fetches the next piece's descriptor, member list and pivot index while it streams the rows of
+// the current one, so the row loads never wait on index loads.  A 16-byte vector of a K row or V
+// row per lane: with D*sizeof(T) = 256 bytes lanes 0-15 carry the K row and lanes 16-31 the V
+// row.  A single-piece slot is finished here (pivot row with weight 1, Eq. 5 weights, normalise,
+// round once); a piece of a multi-piece slot stores its fp32 partial sums for merge_finish_kernel.
 template <typename T>
-__global__ void __launch_bounds__(256) merge_pieces_kernel(const MergeArgs A) {
+__global__ void __launch_bounds__(256) merge_pieces_kernel(const MergeArgs A, int n_uh) {
     constexpr int V = Elem<T>::kVec;
     const int lane = lane_id();
-    const int uh = blockIdx.y, u = uh / A.Hkv, h = uh % A.Hkv;
-    const int piece = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t total = (int64_t)n_uh * A.max_pieces;
     const int rv = A.D / V;                                   // 16-byte vectors per row
-    int slot = piece, first = 0, count = 0, n_pieces = 1, part_base = 0, piece_in_slot = 0;
-    if (A.sorted) {
-        const int *poff = A.piece_off + (int64_t)uh * (A.B + 1);
-        if (piece >= poff[A.B]) return;
-        int a = 0, b = A.B;                                   // largest s with piece_off[s] <= piece
-        while (b - a > 1) {
-            const int mid = (a + b) >> 1;
-            if (poff[mid] <= piece) a = mid; else b = mid;
-        }
-        slot = a;
-        const int *off = A.off + (int64_t)uh * (A.B + 1);
-        const int n = off[slot + 1] - off[slot];
-        n_pieces = poff[slot + 1] - poff[slot];
-        piece_in_slot = piece - poff[slot];
-        first = off[slot] + piece_in_slot * kPiece;
-        count = min(kPiece, n - piece_in_slot * kPiece);
-        part_base = A.part_off[(int64_t)uh * (A.B + 1) + slot];
-    } else if (piece >= A.B) {
-        return;
-    }
-    const T *kb = static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
-    const T *vb = static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1];
-    const int *evi = A.evicted + (int64_t)uh * A.E;
-    const int *sorted = A.sorted ? A.sorted + (int64_t)uh * A.E : nullptr;
-    const float *sim = A.match_sim + (int64_t)uh * A.E;
+    const int n_vec = 2 * rv;
 
-    for (int vec = lane; vec < 2 * rv; vec += 32) {           // which vector of the (K row, V row) pair
-        const bool is_v = vec >= rv;
-        const int c0 = (is_v ? vec - rv : vec) * V;
-        const T *src = is_v ? vb : kb;
-        const int64_t tstride = is_v ? A.vs[2] : A.ks[2];
-        float acc[V];
+    struct Piece { int4 d; int tok_lo, tok_hi, r; float w_lo, w_hi; };
+    auto fetch_desc = [&](int64_t g) -> int4 {               // (slot, first, count, part); count < 0: no such piece
+        if (g >= total) return make_int4(0, 0, -1, -1);
+        if (!A.piece_desc) return make_int4((int)(g % A.max_pieces), 0, 0, -1);      // E == 0: plain copy of the pivots
+        return A.piece_desc[g];
+    };
+    auto fetch_members = [&](int64_t g, Piece &pc) {         // needs pc.d
+        pc.tok_lo = pc.tok_hi = pc.r = 0; pc.w_lo = pc.w_hi = 0.f;
+        if (pc.d.z < 0) return;
+        const int64_t uh = g / A.max_pieces;
+        if (pc.d.z > 0) {
+            const int *mt = A.mem_tok + uh * A.E + pc.d.y;
+            const float *mw = A.mem_w + uh * A.E + pc.d.y;
+            if (lane < pc.d.z) { pc.tok_lo = mt[lane]; pc.w_lo = mw[lane]; }
+            if (lane + 32 < pc.d.z) { pc.tok_hi = mt[lane + 32]; pc.w_hi = mw[lane + 32]; }
+        }
+        if (pc.d.w < 0) pc.r = A.retained[uh * A.B + pc.d.x];
+    };
+
+    int64_t g = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    Piece cur, nxt;
+    cur.d = fetch_desc(g);
+    nxt.d = fetch_desc(g + n_warps);
+    fetch_members(g, cur);
+    for (; g < total; g += n_warps) {
+        const int4 d2 = fetch_desc(g + 2 * n_warps);          // two pieces ahead
+        fetch_members(g + n_warps, nxt);                      // one piece ahead
+        const int slot = cur.d.x, count = cur.d.z, part = cur.d.w;
+        if (count >= 0) {
+            const int uh = (int)(g / A.max_pieces), u = uh / A.Hkv, h = uh % A.Hkv;
+            const T *kb = static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
+            const T *vb = static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1];
+            for (int vec0 = 0; vec0 < n_vec; vec0 += 32) {    // which vector of the (K row, V row) pair
+                const int vec = vec0 + lane;
+                const bool on = vec < n_vec;
+                const bool is_v = vec >= rv;
+                const int c0 = on ? (is_v ? vec - rv : vec) * V : 0;
+                const T *src = is_v ? vb : kb;
+                const int64_t tstride = is_v ? A.vs[2] : A.ks[2];
+                float acc[V];
 #pragma unroll
-        for (int e = 0; e < V; ++e) acc[e] = 0.f;
-        float wsum = 0.f;
-        int t = 0;
-        for (; t + 4 <= count; t += 4) {                      // four rows in flight
-            int j[4]; float w[4]; float x[4][V];
+                for (int e = 0; e < V; ++e) acc[e] = 0.f;
+                float wsum = 0.f;
+                uint4 xr = make_uint4(0, 0, 0, 0);
+                if (on && part < 0) xr = load_raw16(src + (int64_t)cur.r * tstride + c0);    // the pivot row, early
+                for (int t0 = 0; t0 < count; t0 += kMergeBatch) {
+                    uint4 x[kMergeBatch];
+                    int tok[kMergeBatch];
+                    float w[kMergeBatch];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) j[q] = sorted[first + t + q];
+                    for (int q = 0; q < kMergeBatch; ++q) {   // this batch's positions and weights from the lanes that hold them
+                        const int t = t0 + q;
+                        tok[q] = __shfl_sync(0xFFFFFFFFu, t < 32 ? cur.tok_lo : cur.tok_hi, t & 31);
+                        w[q] = __shfl_sync(0xFFFFFFFFu, t < 32 ? cur.w_lo : cur.w_hi, t & 31);
+                    }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                Elem<T>::load16(src + (int64_t)evi[j[q]] * tstride + c0, x[q]);
-                w[q] = A.merge_mode == 1 ? 1.f : __expf(sim[j[q]] - 1.f);
-            }
+                    for (int q = 0; q < kMergeBatch; ++q)     // the batch's row loads, back to back
+                        x[q] = (t0 + q < count && on) ? load_raw16(src + (int64_t)tok[q] * tstride + c0) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                wsum += w[q];
+                    for (int q = 0; q < kMergeBatch; ++q) {   // fixed order: ascending member index
+                        if (t0 + q < count) {
+                            float xf[V];
+                            Elem<T>::unpack(x[q], xf);
+                            wsum += w[q];
 #pragma unroll
-                for (int e = 0; e < V; ++e) acc[e] = fmaf(w[q], x[q][e], acc[e]);
+                            for (int e = 0; e < V; ++e) acc[e] = fmaf(w[q], xf[e], acc[e]);
+                        }
+                    }
+                }
+                if (!on) continue;
+                if (part < 0) {
+                    T *dst = is_v ? static_cast<T *>(A.v_out) + u * A.vos[0] + h * A.vos[1] + (int64_t)slot * A.vos[2]
+                                  : static_cast<T *>(A.k_out) + u * A.kos[0] + h * A.kos[1] + (int64_t)slot * A.kos[2];
+                    if (count == 0) {
+                        *reinterpret_cast<uint4 *>(dst + c0) = xr;   // nothing merged in: the pivot row, bit for bit
+                    } else {
+                        const float inv = 1.f / (1.f + wsum);
+                        float xf[V], o[V];
+                        Elem<T>::unpack(xr, xf);
+#pragma unroll
+                        for (int e = 0; e < V; ++e) o[e] = (xf[e] + acc[e]) * inv;
+                        Elem<T>::store16(dst + c0, o);
+                    }
+                } else {
+                    float *rec = A.partial + ((int64_t)uh * A.max_parts + part) * (2 * A.D + 4);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) rec[(is_v ? A.D : 0) + c0 + e] = acc[e];
+                    if (vec == 0) rec[2 * A.D] = wsum;
+                }
             }
         }
-        for (; t < count; ++t) {
-            const int j = sorted[first + t];
-            float x[V];
-            Elem<T>::load16(src + (int64_t)evi[j] * tstride + c0, x);
-            const float w = A.merge_mode == 1 ? 1.f : __expf(sim[j] - 1.f);
-            wsum += w;
-#pragma unroll
-            for (int e = 0; e < V; ++e) acc[e] = fmaf(w, x[e], acc[e]);
-        }
-        if (n_pieces == 1) {
-            const int r = A.retained[(int64_t)uh * A.B + slot];
-            float x[V];
-            Elem<T>::load16(src + (int64_t)r * tstride + c0, x);
-            T *dst = is_v ? static_cast<T *>(A.v_out) + u * A.vos[0] + h * A.vos[1] + (int64_t)slot * A.vos[2]
-                          : static_cast<T *>(A.k_out) + u * A.kos[0] + h * A.kos[1] + (int64_t)slot * A.kos[2];
-            if (count == 0) {
-                Elem<T>::store16(dst + c0, x);                // nothing merged in: the pivot row, bit for bit
-            } else {
-                const float inv = 1.f / (1.f + wsum);
-                float o[V];
-#pragma unroll
-                for (int e = 0; e < V; ++e) o[e] = (x[e] + acc[e]) * inv;
-                Elem<T>::store16(dst + c0, o);
-            }
-        } else {
-            float *rec = A.partial + ((int64_t)uh * A.max_parts + part_base + piece_in_slot) * (2 * A.D + 4);
-#pragma unroll
-            for (int e = 0; e < V; ++e) rec[(is_v ? A.D : 0) + c0 + e] = acc[e];
-            if (vec == 0) rec[2 * A.D] = wsum;
-        }
+        cur = nxt;
+        nxt.d = d2;
     }
 }
 

@@ -64,7 +64,9 @@ struct Ctx {
     }
 };
 
-__device__ __forceinline__ Ctx setup(uint8_t *smem_raw, const CUtensorMap *ma, const CUtensorMap *mb, int *status) {
+// `a_readers`: epilogue warps per half that read the A stage themselves and release it with a_release().
+__device__ __forceinline__ Ctx setup(uint8_t *smem_raw, const CUtensorMap *ma, const CUtensorMap *mb, int *status,
+                                     int a_readers = 0) {
     Ctx c;
     c.base = tc::smem_u32(smem_raw);
     c.gen = smem_raw;
@@ -82,7 +84,7 @@ __device__ __forceinline__ Ctx setup(uint8_t *smem_raw, const CUtensorMap *ma, c
     }
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(c.gen + kSmemBar + 128);
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 10; ++i) tc::mbar_init(c.bar(i), 1);
+        for (int i = 0; i < 10; ++i) tc::mbar_init(c.bar(i), (i == 2 || i == 3) ? 1 + a_readers : 1);
         tc::mbar_init(c.bar(10), 4);           // one arrival per epilogue warp of the half
         tc::mbar_init(c.bar(11), 4);
         for (int i = 12; i < 16; ++i) tc::mbar_init(c.bar(i), 1);
@@ -197,6 +199,15 @@ __device__ __forceinline__ bool acc_wait(const Ctx &c, int k, int *status) {
     const bool ok = tc::mbar_wait(c.bar(8 + c.group), k & 1, c.abort_flag, status);
     tc::tc_fence_after();
     return ok;
+}
+// For kernels whose epilogue reads its A half from shared memory: wait until the half of the
+// n-th item this group takes part in has landed / hand it back (one arrival per warp).
+__device__ __forceinline__ bool a_wait(const Ctx &c, int n, int *status) {
+    return tc::mbar_wait(c.bar(c.group), n & 1, c.abort_flag, status);
+}
+__device__ __forceinline__ void a_release(const Ctx &c) {
+    __syncwarp();
+    if (c.lane == 0) tc::mbar_arrive(c.bar(2 + c.group));
 }
 // Waits until the per-column constants of the bt-th B tile are in shared memory.
 __device__ __forceinline__ bool extra_wait(const Ctx &c, int bt, int *status) {
