@@ -167,7 +167,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         if (c.lane == 0) tcs::mma_issuer(c, A.n_items, plan, A.status);
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
-        float4 *wrow = reinterpret_cast<float4 *>(c.epi_scratch()) + row * 4;   // 16 floats per row
+        float4 *wrow = reinterpret_cast<float4 *>(c.epi_scratch()) + row * 2;          // 8 floats per row
+        float4 *prow = reinterpret_cast<float4 *>(c.partner_scratch()) + row * 2;      // the other column half's
         int k = 0, bt = 0, n_mine = 0;
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
@@ -186,23 +187,24 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             if (!active) {
                 if (!p.tp.empty()) bt += p.tp.n_tiles;               // keep the B-tile count in step
             } else {
-                // the token's key row sits in this half's A stage (128-byte rows, 16-byte units XOR-swizzled by
-                // the row index): read it once for the norm while the first MMAs run, then hand the stage back
-                ok = tcs::a_wait(c, n_mine++, A.status);
-                if (!ok) break;
-                const uint8_t *a_half = c.gen + tcs::kSmemA + c.group * tcs::kAHalf + row * 128;
+                if (c.colhalf == 0) {
+                    // the token's key row sits in this half's A stage (128-byte rows, 16-byte units XOR-swizzled by
+                    // the row index): read it once for the norm while the first MMAs run, then hand the stage back
+                    ok = tcs::a_wait(c, n_mine++, A.status);
+                    const uint8_t *a_half = c.gen + tcs::kSmemA + c.group * tcs::kAHalf + row * 128;
 #pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {
+                    for (int kh = 0; kh < 2; ++kh) {
 #pragma unroll
-                    for (int un = 0; un < 8; ++un) {
-                        const uint4 raw = *reinterpret_cast<const uint4 *>(a_half + kh * (tcs::kAHalf / 2) + ((un ^ (row & 7)) << 4));
-                        float x[8];
-                        Elem<__nv_bfloat16>::unpack(raw, x);
+                        for (int un = 0; un < 8; ++un) {
+                            const uint4 raw = *reinterpret_cast<const uint4 *>(a_half + kh * (tcs::kAHalf / 2) + ((un ^ (row & 7)) << 4));
+                            float x[8];
+                            Elem<__nv_bfloat16>::unpack(raw, x);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
+                            for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
+                        }
                     }
+                    tcs::a_release(c);
                 }
-                tcs::a_release(c);
                 for (int t = 0; ok && t < p.tp.n_tiles; ++t, ++k, ++bt) {
                     const int col0 = p.lo + t * kMtCols;
                     const int ncols = min(kMtCols, p.hi - col0);
@@ -228,51 +230,62 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                                 v[j] = valid ? v[j] : -INFINITY;
                             }
                         }
-                        float lo5[5], hi5[5];
+                        float q8[4];                         // maxima of the four groups of 8 columns
 #pragma unroll
-                        for (int i = 0; i < 5; ++i) {
-                            lo5[i] = tc::max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-                            hi5[i] = tc::max3(v[16 + 3 * i], v[17 + 3 * i], v[18 + 3 * i]);
-                        }
-                        const float lo = tc::max3(tc::max3(lo5[0], lo5[1], lo5[2]), tc::max3(lo5[3], lo5[4], v[15]), -INFINITY);
-                        const float hi = tc::max3(tc::max3(hi5[0], hi5[1], hi5[2]), tc::max3(hi5[3], hi5[4], v[31]), -INFINITY);
+                        for (int g = 0; g < 4; ++g)
+                            q8[g] = tc::max3(tc::max3(v[8 * g], v[8 * g + 1], v[8 * g + 2]),
+                                             tc::max3(v[8 * g + 3], v[8 * g + 4], v[8 * g + 5]),
+                                             tc::max3(v[8 * g + 6], v[8 * g + 7], -INFINITY));   // never NaN: the comparisons below are safe
+                        const float lo = fmaxf(q8[0], q8[1]), hi = fmaxf(q8[2], q8[3]);
                         const float cmax = fmaxf(lo, hi);
                         if (cmax > best) {                           // strict: an earlier chunk keeps a tie
                             best = cmax;
-                            const bool low = lo >= hi;               // a tie between the halves goes to the lower columns
-                            best_cc = low ? cc : cc + 16;
+                            const bool low = lo >= hi;               // ties between groups go to the lower columns
+                            const bool first = low ? q8[0] >= q8[1] : q8[2] >= q8[3];
+                            best_cc = cc + (low ? 0 : 16) + (first ? 0 : 8);
+                            float w16[16];
 #pragma unroll
-                            for (int q4 = 0; q4 < 4; ++q4)           // keep the 16 columns to find the exact one later
-                                wrow[q4] = low ? make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3])
-                                               : make_float4(v[16 + 4 * q4], v[17 + 4 * q4], v[18 + 4 * q4], v[19 + 4 * q4]);
+                            for (int i = 0; i < 16; ++i) w16[i] = low ? v[i] : v[16 + i];
+                            wrow[0] = first ? make_float4(w16[0], w16[1], w16[2], w16[3]) : make_float4(w16[8], w16[9], w16[10], w16[11]);
+                            wrow[1] = first ? make_float4(w16[4], w16[5], w16[6], w16[7]) : make_float4(w16[12], w16[13], w16[14], w16[15]);
                         }
                     });
                     tcs::acc_release(c);
                 }
             }
-            if (!ok) break;
-            if (in_range) {
-                const int j = A.rank[(int64_t)p.uh * A.L + token];
-                if (j >= 0) {                                        // a non-pivot: report its match
-                    int slot = -1;
-                    float sim = 0.f;
-                    if (best_cc >= 0) {
-                        int idx = 0;
+            // (after a wait that ran out the results are garbage, but the two meeting points below are still
+            // kept so that the partner warp is never left waiting; the loop ends right after them)
+            // this warp's result for the row: similarity (still times the row's norm) and pivot slot
+            int slot = -1;
+            if (best_cc >= 0 && ok) {
+                int idx = 0;
 #pragma unroll
-                        for (int q4 = 3; q4 >= 0; --q4) {            // lowest column that holds the maximum
-                            const float4 w = wrow[q4];
-                            if (w.w == best) idx = 4 * q4 + 3;
-                            if (w.z == best) idx = 4 * q4 + 2;
-                            if (w.y == best) idx = 4 * q4 + 1;
-                            if (w.x == best) idx = 4 * q4;
-                        }
-                        slot = A.cand_slot[(int64_t)p.uh * A.Ctot + best_cc + idx];
-                        sim = ssq > 0.f ? best * rsqrtf(ssq) : 0.f;
+                for (int q4 = 1; q4 >= 0; --q4) {                    // lowest column that holds the maximum
+                    const float4 w = wrow[q4];
+                    if (w.w == best) idx = 4 * q4 + 3;
+                    if (w.z == best) idx = 4 * q4 + 2;
+                    if (w.y == best) idx = 4 * q4 + 1;
+                    if (w.x == best) idx = 4 * q4;
+                }
+                slot = A.cand_slot[(int64_t)p.uh * A.Ctot + best_cc + idx];
+            }
+            // the upper column half hands its result to the lower one, which owns the row's output
+            if (c.colhalf == 1) wrow[0] = make_float4(best, __int_as_float(slot), 0.f, 0.f);
+            tcs::pair_sync(c);
+            if (c.colhalf == 0 && ok) {
+                const float4 other = prow[0];
+                if (other.x > best) { best = other.x; slot = __float_as_int(other.y); }    // a tie stays with the lower columns
+                if (in_range) {
+                    const int j = A.rank[(int64_t)p.uh * A.L + token];
+                    if (j >= 0) {                                    // a non-pivot: report its match
+                        float sim = 0.f;
+                        if (slot >= 0 && ssq > 0.f) sim = best * rsqrtf(ssq);
+                        A.match[(int64_t)p.uh * A.E + j] = slot;
+                        A.match_sim[(int64_t)p.uh * A.E + j] = sim;
                     }
-                    A.match[(int64_t)p.uh * A.E + j] = slot;
-                    A.match_sim[(int64_t)p.uh * A.E + j] = sim;
                 }
             }
+            tcs::pair_sync(c);                                       // the hand-over slot may be overwritten again
         }
     }
     tcs::teardown(c);

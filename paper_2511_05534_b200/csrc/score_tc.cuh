@@ -19,7 +19,7 @@
 namespace flowmm {
 
 struct ScoreTcArgs {
-    float2 *row_part;            // [UH*GW, n_chunk] (max, sum) per proxy row and key chunk, log2 domain
+    float2 *row_part;            // [UH*GW, 2*n_chunk] (max, sum) per proxy row, key chunk and column half, log2 domain
     float *negc;                 // [UH, GWpad] -(row max + log2 row sum); very negative for padding rows
     const uint8_t *modality;     // [U, L]
     float *importance;           // [UH, L]
@@ -132,7 +132,7 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
                 tcs::acc_release(c);
             }
             if (!ok) break;
-            if (valid_row) A.row_part[((int64_t)uh * A.GW + r) * A.n_chunk + kc] = make_float2(m, l);
+            if (valid_row) A.row_part[((int64_t)uh * A.GW + r) * (2 * A.n_chunk) + 2 * kc + c.colhalf] = make_float2(m, l);
         }
     }
     tcs::teardown(c);
@@ -183,7 +183,9 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
     } else if (c.warp == 1) {
         if (c.lane == 0) tcs::mma_issuer(c, A.n_items2, plan, A.status);
     } else {
-        const int lane = c.lane;
+        const int lane = c.lane, row = c.quarter * 32 + lane;
+        float *xch = reinterpret_cast<float *>(c.epi_scratch()) + row;          // hand-over slot of this row
+        const float *pxch = reinterpret_cast<const float *>(c.partner_scratch()) + row;
         int k = 0, bt = 0, cached_u = -1;
         uint32_t wbits[4] = {0, 0, 0, 0};                            // modality of the proxy tokens, 32 per word
         bool ok = true;
@@ -207,24 +209,25 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                 cached_u = u;
             }
             const int key0 = kt * tcs::kItemRows + c.group * tcs::kRows;
-            const int key = key0 + c.quarter * 32 + lane;
+            const int key = key0 + row;
             const bool masked_tile = key0 + tcs::kRows > A.L - A.W + 1;   // some (key, proxy row) pair is masked
             const bool my_vis = key < A.L && A.modality[(int64_t)u * A.L + key] != 0;
             const int first_proxy = A.L - A.W;
             float imp = 0.f, cg = 0.f;
-            int cur_g = 0;
+            int cur_g = -1;                                          // head whose mass is being summed; -1: none yet
             for (int t = 0; ok && t < p.n_tiles; ++t, ++k, ++bt) {
                 const int ncols = min(tcs::kCols, A.GW - t * tcs::kCols);
-                const int n_chunks = (ncols + 31) >> 5;
                 ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
                 if (!ok) break;
                 const float4 *negc4 = c.extra(bt);
-                tcs::for_each_chunk(c, n_chunks, [&](int ch, uint32_t (&acc)[32]) {
+                tcs::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
                     const int col = t * tcs::kCols + ch * 32;        // proxy row index r = g_local * W + a
                     const int g_local = col / A.W, a0 = col % A.W;
                     if (g_local != cur_g) {                          // a head is complete: publish its mass
-                        const float tot = warp_sum(cg);
-                        if (lane == 0) cross_out[(int64_t)cur_g * (A.n_rt * 8)] = tot;
+                        if (cur_g >= 0) {
+                            const float tot = warp_sum(cg);
+                            if (lane == 0) cross_out[(int64_t)cur_g * (A.n_rt * 8)] = tot;
+                        }
                         cg = 0.f;
                         cur_g = g_local;
                     }
@@ -259,12 +262,16 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                 });
                 tcs::acc_release(c);
             }
-            if (!ok) break;
-            {
+            if (ok && cur_g >= 0) {
                 const float tot = warp_sum(cg);
                 if (lane == 0) cross_out[(int64_t)cur_g * (A.n_rt * 8)] = tot;
             }
-            if (key < A.L) A.importance[(int64_t)uh * A.L + key] = imp / (float)A.G;     // group mean
+            // the two column halves of a key meet: the upper one hands its partial sum over (kept even after a
+            // wait ran out, so that the partner warp is never left waiting)
+            if (c.colhalf == 1) *xch = imp;
+            tcs::pair_sync(c);
+            if (c.colhalf == 0 && ok && key < A.L) A.importance[(int64_t)uh * A.L + key] = (imp + *pxch) / (float)A.G;   // group mean
+            tcs::pair_sync(c);
         }
     }
     tcs::teardown(c);

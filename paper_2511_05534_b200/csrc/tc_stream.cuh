@@ -5,9 +5,11 @@
 // B_0 .. B_{n-1}; every B tile is used by both halves, which halves the operand traffic per
 // multiply-add, and yields one 128 x 256 fp32 accumulator per half in TMEM (half h owns TMEM
 // columns [256 h, 256 h + 256)).
-// Roles: warp 0 issues the TMA loads, warp 1 issues tcgen05.mma, warps 2-5 run the kernel's
-// epilogue on the accumulators of half 0 and warps 6-9 on those of half 1 (two epilogue warps per
-// SM sub-partition, so one half's TMEM reads and arithmetic hide the other's latencies).
+// Roles: warp 0 issues the TMA loads, warp 1 issues tcgen05.mma, warps 2-17 run the kernel's
+// epilogue: a quad of warps (one per 32 TMEM lanes) per (A half, column half), i.e. four epilogue
+// warps per SM sub-partition, so that TMEM reads, shared-memory reads and dependent arithmetic of
+// one warp are covered by the other three.  The two quads of a half split each accumulator's
+// 256 columns (0-127 / 128-255) and combine per-row results through shared memory.
 // Shared-memory stages (one per A half, two for B) and the two accumulators are handed around
 // with mbarriers; every wait is bounded.
 #pragma once
@@ -19,7 +21,7 @@ namespace tcs {
 constexpr int kRows = 128;                   // rows of an A half (UMMA M)
 constexpr int kCols = 256;                   // rows of a B tile (UMMA N)
 constexpr int kItemRows = 2 * kRows;         // rows of A an item covers
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t kAHalf = kRows * 128 * 2;             // bytes of an A half: two 64-element K halves
 constexpr uint32_t kBStage = kCols * 128 * 2;
@@ -53,11 +55,18 @@ struct Ctx {
     volatile int *abort_flag;
     int warp, lane;
     int group, quarter;        // epilogue warps: which A half they serve, which 32 TMEM lanes they read
+    int colhalf;               // ... and which 128 columns of each accumulator
     bool ok;                   // false: shared memory was not 1024-byte aligned; nothing may run
     // barrier slots: 0-1 a_full[h], 2-3 a_empty[h], 4-5 b_full[s], 6-7 b_empty[s], 8-9 acc_full[h], 10-11 acc_empty[h],
     // 12-15 x_full[slot] (per-column constants landed)
     __device__ __forceinline__ uint32_t bar(int i) const { return bars + 8u * i; }
-    __device__ __forceinline__ uint8_t *epi_scratch() const { return gen + kSmemEpi + (uint32_t)group * (kEpiBytes / 2); }
+    // scratch of this warp's quad (a quarter of the epilogue scratch) / of its partner quad on the same rows
+    __device__ __forceinline__ uint8_t *epi_scratch() const {
+        return gen + kSmemEpi + (uint32_t)(group * 2 + colhalf) * (kEpiBytes / 4);
+    }
+    __device__ __forceinline__ uint8_t *partner_scratch() const {
+        return gen + kSmemEpi + (uint32_t)(group * 2 + (colhalf ^ 1)) * (kEpiBytes / 4);
+    }
     // per-column constants of the bt-th B tile this CTA streams (valid from the tile's acc_wait to its release)
     __device__ __forceinline__ const float4 *extra(int bt) const {
         return reinterpret_cast<const float4 *>(gen + kSmemExtra + (uint32_t)(bt & (kExtraSlots - 1)) * kExtraBytes);
@@ -73,8 +82,9 @@ __device__ __forceinline__ Ctx setup(uint8_t *smem_raw, const CUtensorMap *ma, c
     c.bars = c.base + kSmemBar;
     c.warp = threadIdx.x >> 5;
     c.lane = threadIdx.x & 31;
-    c.group = c.warp >= 6 ? 1 : 0;
+    c.group = ((c.warp - 2) >> 2) & 1;
     c.quarter = c.warp & 3;
+    c.colhalf = (c.warp - 2) >> 3;
     c.tmem_base = 0;
     c.abort_flag = reinterpret_cast<volatile int *>(c.gen + kSmemBar + 132);
     c.ok = (c.base & 1023u) == 0;              // the swizzled operand tiles need a 1024-byte aligned base
@@ -85,8 +95,8 @@ __device__ __forceinline__ Ctx setup(uint8_t *smem_raw, const CUtensorMap *ma, c
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(c.gen + kSmemBar + 128);
     if (threadIdx.x == 0) {
         for (int i = 0; i < 10; ++i) tc::mbar_init(c.bar(i), (i == 2 || i == 3) ? 1 + a_readers : 1);
-        tc::mbar_init(c.bar(10), 4);           // one arrival per epilogue warp of the half
-        tc::mbar_init(c.bar(11), 4);
+        tc::mbar_init(c.bar(10), 8);           // one arrival per epilogue warp of the half
+        tc::mbar_init(c.bar(11), 8);
         for (int i = 12; i < 16; ++i) tc::mbar_init(c.bar(i), 1);
         *c.abort_flag = 0;
         tc::mbar_init_fence();
@@ -223,23 +233,21 @@ __device__ __forceinline__ uint32_t acc_addr(const Ctx &c, int chunk) {
     return c.tmem_base + c.group * kCols + chunk * 32 + ((uint32_t)(c.quarter * 32) << 16);
 }
 
-// Runs f(chunk, values) over the first n_chunks 32-column chunks of the current accumulator with the
-// TMEM load of chunk i+1 in flight while chunk i is processed.
+// Runs f(chunk, values) over this warp's 32-column chunks of the current accumulator: chunks
+// 4*colhalf .. 4*colhalf+3, as far as they lie below n_chunks (the tile's chunk count).
 template <class F>
 __device__ __forceinline__ void for_each_chunk(const Ctx &c, int n_chunks, F &&f) {
-    uint32_t a[32], b[32];
-    if (n_chunks <= 0) return;
-    tc::tmem_ld32(acc_addr(c, 0), a);
-    for (int ch = 0; ch < n_chunks; ch += 2) {
+    const int hi = min(n_chunks, 4 * c.colhalf + 4);
+    for (int ch = 4 * c.colhalf; ch < hi; ++ch) {
+        uint32_t a[32];
+        tc::tmem_ld32(acc_addr(c, ch), a);
         tc::tmem_ld_wait(a);
-        if (ch + 1 < n_chunks) tc::tmem_ld32(acc_addr(c, ch + 1), b);
         f(ch, a);
-        if (ch + 1 < n_chunks) {
-            tc::tmem_ld_wait(b);
-            if (ch + 2 < n_chunks) tc::tmem_ld32(acc_addr(c, ch + 2), a);
-            f(ch + 1, b);
-        }
     }
+}
+// Meeting point of the two warps that share rows (same half, same lanes, other columns).
+__device__ __forceinline__ void pair_sync(const Ctx &c) {
+    asm volatile("bar.sync %0, 64;" ::"r"(1 + c.group * 4 + c.quarter) : "memory");
 }
 
 }  // namespace tcs
