@@ -107,6 +107,26 @@ class ClockSampler:
         return out
 
 
+def match_pair_count(p, tau_eff, diag, modality):
+    """Number of (non-pivot, admissible pivot) pairs whose similarity Eq. 9-10 need, summed over
+    all units and heads: the gate of Eq. 10 removes pivots above tau, an intra-modal layer pairs
+    tokens of equal modality only.  Counted from one call's own outputs; accounting only."""
+    import torch
+    imp, ret, strat = diag["importance"], diag["retained"].long(), diag["strategy"]
+    U, Hkv, L = imp.shape
+    mod = modality.bool()[:, None, :].expand(U, Hkv, L)
+    adm = torch.gather(imp, 2, ret) <= tau_eff
+    ret_vis = torch.gather(mod, 2, ret)
+    n_v = (adm & ret_vis).sum(-1).double()
+    n_t = (adm & ~ret_vis).sum(-1).double()
+    tot_vis = modality.bool().sum(-1).double()[:, None]
+    e_v = tot_vis - ret_vis.sum(-1).double()
+    e_t = (L - tot_vis) - (~ret_vis).sum(-1).double()
+    cross = (strat == 1).double()[:, None]
+    pairs = cross * (e_t + e_v) * (n_t + n_v) + (1 - cross) * (e_t * n_t + e_v * n_v)
+    return float(pairs.sum().item())
+
+
 def kernel_model(wl, B, dsize):
     """Algorithmic flops and bytes of each kernel for ONE unit (all heads), from the
     operation's definition: what must be read and written once, and the multiply-adds of the
@@ -290,11 +310,20 @@ def run_ours(args):
     torch.cuda.synchronize()
     peaks = load_peaks()
     model = kernel_model(wl, B, dsize)
+    # the match step's own flops: only pairs that pass the gates of Eq. 10 need a similarity
+    tau_eff = wl.tau_rel * wl.window / wl.seq_len
+    q0, k0, v0, m0 = sets[0]
+    diag = F.compress_layer_alloc(p, q0, k0, v0, m0, ws=ws)
+    pairs = match_pair_count(p, tau_eff, diag, m0)
+    dense_pairs = float(U) * wl.n_kv_heads * (wl.seq_len - B) * B
+    del diag
     kernels = {}
     for name, times in per_kernel.items():
         avg = sum(times) / len(times)
         flops, nbytes = model_for(name, model)
         flops, nbytes = flops * U, nbytes * U
+        if KERNEL_MODEL.get(name) == "match":
+            flops = 2.0 * wl.head_dim * pairs
         t_tensor = flops / (peaks["bf16_tflops_sustained"] * 1e12) if dt_code == F.BF16 else 0.0
         t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
         bound = "tensor" if t_tensor > t_hbm else "hbm"
@@ -345,7 +374,8 @@ def run_ours(args):
             "config": {"workload": wl.name, "layers": n_layers, "seqs": wl.n_seqs, "n_q_heads": wl.n_q_heads,
                        "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "seq_len": wl.seq_len,
                        "window": wl.window, "budget_permille": args.permille, "n_keep": B,
-                       "units_per_call": U, "l2": "%d rotating input sets of %.0f MB (inputs larger than L2)" %
+                       "units_per_call": U, "match_pairs_fraction_of_dense": round(pairs / max(1.0, dense_pairs), 4),
+                       "l2": "%d rotating input sets of %.0f MB (inputs larger than L2)" %
                        (n_sets, bytes_per_set / 1e6), "path": args.path, "parallelism": "units sharded, no collective"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

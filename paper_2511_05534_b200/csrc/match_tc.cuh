@@ -10,6 +10,8 @@
 // norms enter in fp32 afterwards, so no precision is lost before the argmax.
 // An intra-modal layer visits only the candidate group of the row tile's modality.
 #pragma once
+#include <type_traits>
+
 #include "common.cuh"
 #include "tc_stream.cuh"
 
@@ -167,8 +169,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         if (c.lane == 0) tcs::mma_issuer(c, A.n_items, plan, A.status);
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
-        float4 *wrow = reinterpret_cast<float4 *>(c.epi_scratch()) + row * 2;          // 8 floats per row
-        float4 *prow = reinterpret_cast<float4 *>(c.partner_scratch()) + row * 2;      // the other column half's
+        const uint32_t wrow = c.epi_addr() + row * 32;          // 8 floats per row
+        const uint32_t prow = c.partner_addr() + row * 32;      // the other column half's
         int k = 0, bt = 0, n_mine = 0;
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
@@ -191,12 +193,14 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     // the token's key row sits in this half's A stage (128-byte rows, 16-byte units XOR-swizzled by
                     // the row index): read it once for the norm while the first MMAs run, then hand the stage back
                     ok = tcs::a_wait(c, n_mine++, A.status);
-                    const uint8_t *a_half = c.gen + tcs::kSmemA + c.group * tcs::kAHalf + row * 128;
+                    const uint32_t a_half = c.base + tcs::kSmemA + c.group * tcs::kAHalf + row * 128;
 #pragma unroll
                     for (int kh = 0; kh < 2; ++kh) {
 #pragma unroll
                         for (int un = 0; un < 8; ++un) {
-                            const uint4 raw = *reinterpret_cast<const uint4 *>(a_half + kh * (tcs::kAHalf / 2) + ((un ^ (row & 7)) << 4));
+                            const float4 rawf = tc::lds128(a_half + kh * (tcs::kAHalf / 2) + ((un ^ (row & 7)) << 4));
+                            const uint4 raw = make_uint4(__float_as_uint(rawf.x), __float_as_uint(rawf.y), __float_as_uint(rawf.z),
+                                                         __float_as_uint(rawf.w));
                             float x[8];
                             Elem<__nv_bfloat16>::unpack(raw, x);
 #pragma unroll
@@ -210,19 +214,21 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     const int ncols = min(kMtCols, p.hi - col0);
                     ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
                     if (!ok) break;
-                    const float4 *scale4 = c.extra(bt);              // reciprocal norms of this tile's candidates
-                    tcs::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
+                    const uint32_t scale4 = c.extra(bt);             // reciprocal norms of this tile's candidates
+                    // one chunk of 32 columns; kMasked: rows of the tile differ in which columns they may take
+                    auto chunk = [&](auto masked_tag, int ch, uint32_t (&acc)[32]) {
+                        constexpr bool kMasked = decltype(masked_tag)::value;
                         const int cc = col0 + ch * 32;
                         float v[32];
 #pragma unroll
                         for (int q4 = 0; q4 < 8; ++q4) {     // a column that is no candidate has scale NaN and never wins
-                            const float4 s4 = scale4[ch * 8 + q4];
+                            const float4 s4 = tc::lds128(scale4 + (ch * 8 + q4) * 16);
                             v[4 * q4 + 0] = __uint_as_float(acc[4 * q4 + 0]) * s4.x;
                             v[4 * q4 + 1] = __uint_as_float(acc[4 * q4 + 1]) * s4.y;
                             v[4 * q4 + 2] = __uint_as_float(acc[4 * q4 + 2]) * s4.z;
                             v[4 * q4 + 3] = __uint_as_float(acc[4 * q4 + 3]) * s4.w;
                         }
-                        if (row_masked) {                    // intra-modal layer, tile with tokens of both modalities
+                        if constexpr (kMasked) {             // intra-modal layer, tile with tokens of both modalities
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
                                 const int col = cc + j;
@@ -230,26 +236,25 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                                 v[j] = valid ? v[j] : -INFINITY;
                             }
                         }
-                        float q8[4];                         // maxima of the four groups of 8 columns
 #pragma unroll
-                        for (int g = 0; g < 4; ++g)
-                            q8[g] = tc::max3(tc::max3(v[8 * g], v[8 * g + 1], v[8 * g + 2]),
-                                             tc::max3(v[8 * g + 3], v[8 * g + 4], v[8 * g + 5]),
-                                             tc::max3(v[8 * g + 6], v[8 * g + 7], -INFINITY));   // never NaN: the comparisons below are safe
-                        const float lo = fmaxf(q8[0], q8[1]), hi = fmaxf(q8[2], q8[3]);
-                        const float cmax = fmaxf(lo, hi);
-                        if (cmax > best) {                           // strict: an earlier chunk keeps a tie
-                            best = cmax;
-                            const bool low = lo >= hi;               // ties between groups go to the lower columns
-                            const bool first = low ? q8[0] >= q8[1] : q8[2] >= q8[3];
-                            best_cc = cc + (low ? 0 : 16) + (first ? 0 : 8);
-                            float w16[16];
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) w16[i] = low ? v[i] : v[16 + i];
-                            wrow[0] = first ? make_float4(w16[0], w16[1], w16[2], w16[3]) : make_float4(w16[8], w16[9], w16[10], w16[11]);
-                            wrow[1] = first ? make_float4(w16[4], w16[5], w16[6], w16[7]) : make_float4(w16[12], w16[13], w16[14], w16[15]);
+                        for (int g = 0; g < 4; ++g) {        // four groups of 8 columns, in column order
+                            const float q8 = tc::max3(tc::max3(v[8 * g], v[8 * g + 1], v[8 * g + 2]),
+                                                      tc::max3(v[8 * g + 3], v[8 * g + 4], v[8 * g + 5]),
+                                                      fmaxf(v[8 * g + 6], v[8 * g + 7]));
+                            if (q8 > best) {                 // strict: an earlier group keeps a tie (false for NaN)
+                                best = q8;
+                                best_cc = cc + 8 * g;
+                                // keep the 8 columns to find the exact one later
+                                tc::sts128(wrow, v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3]);
+                                tc::sts128(wrow + 16, v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]);
+                            }
                         }
-                    });
+                    };
+                    const int n_chunks = (ncols + 31) >> 5;
+                    if (row_masked)
+                        tcs::for_each_chunk(c, n_chunks, [&](int ch, uint32_t (&acc)[32]) { chunk(std::true_type{}, ch, acc); });
+                    else
+                        tcs::for_each_chunk(c, n_chunks, [&](int ch, uint32_t (&acc)[32]) { chunk(std::false_type{}, ch, acc); });
                     tcs::acc_release(c);
                 }
             }
@@ -261,7 +266,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 int idx = 0;
 #pragma unroll
                 for (int q4 = 1; q4 >= 0; --q4) {                    // lowest column that holds the maximum
-                    const float4 w = wrow[q4];
+                    const float4 w = tc::lds128(wrow + q4 * 16);
                     if (w.w == best) idx = 4 * q4 + 3;
                     if (w.z == best) idx = 4 * q4 + 2;
                     if (w.y == best) idx = 4 * q4 + 1;
@@ -270,10 +275,10 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 slot = A.cand_slot[(int64_t)p.uh * A.Ctot + best_cc + idx];
             }
             // the upper column half hands its result to the lower one, which owns the row's output
-            if (c.colhalf == 1) wrow[0] = make_float4(best, __int_as_float(slot), 0.f, 0.f);
+            if (c.colhalf == 1) tc::sts128(wrow, best, __int_as_float(slot), 0.f, 0.f);
             tcs::pair_sync(c);
             if (c.colhalf == 0 && ok) {
-                const float4 other = prow[0];
+                const float4 other = tc::lds128(prow);
                 if (other.x > best) { best = other.x; slot = __float_as_int(other.y); }    // a tie stays with the lower columns
                 if (in_range) {
                     const int j = A.rank[(int64_t)p.uh * A.L + token];

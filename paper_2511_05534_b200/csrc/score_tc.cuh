@@ -184,8 +184,8 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
         if (c.lane == 0) tcs::mma_issuer(c, A.n_items2, plan, A.status);
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
-        float *xch = reinterpret_cast<float *>(c.epi_scratch()) + row;          // hand-over slot of this row
-        const float *pxch = reinterpret_cast<const float *>(c.partner_scratch()) + row;
+        const uint32_t xch = c.epi_addr() + row * 4;            // hand-over slot of this row
+        const uint32_t pxch = c.partner_addr() + row * 4;
         int k = 0, bt = 0, cached_u = -1;
         uint32_t wbits[4] = {0, 0, 0, 0};                            // modality of the proxy tokens, 32 per word
         bool ok = true;
@@ -219,7 +219,7 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                 const int ncols = min(tcs::kCols, A.GW - t * tcs::kCols);
                 ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
                 if (!ok) break;
-                const float4 *negc4 = c.extra(bt);
+                const uint32_t negc4 = c.extra(bt);
                 tcs::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
                     const int col = t * tcs::kCols + ch * 32;        // proxy row index r = g_local * W + a
                     const int g_local = col / A.W, a0 = col % A.W;
@@ -234,7 +234,7 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                     float pr[32];
 #pragma unroll
                     for (int q4 = 0; q4 < 8; ++q4) {
-                        const float4 n4 = negc4[ch * 8 + q4];
+                        const float4 n4 = tc::lds128(negc4 + (ch * 8 + q4) * 16);
                         pr[4 * q4 + 0] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 0]), A.scale_log2, n4.x));
                         pr[4 * q4 + 1] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 1]), A.scale_log2, n4.y));
                         pr[4 * q4 + 2] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 2]), A.scale_log2, n4.z));
@@ -268,9 +268,9 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
             }
             // the two column halves of a key meet: the upper one hands its partial sum over (kept even after a
             // wait ran out, so that the partner warp is never left waiting)
-            if (c.colhalf == 1) *xch = imp;
+            if (c.colhalf == 1) tc::sts32(xch, imp);
             tcs::pair_sync(c);
-            if (c.colhalf == 0 && ok && key < A.L) A.importance[(int64_t)uh * A.L + key] = (imp + *pxch) / (float)A.G;   // group mean
+            if (c.colhalf == 0 && ok && key < A.L) A.importance[(int64_t)uh * A.L + key] = (imp + tc::lds32(pxch)) / (float)A.G;   // group mean
             tcs::pair_sync(c);
         }
     }

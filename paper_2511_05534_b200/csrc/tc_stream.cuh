@@ -67,9 +67,15 @@ struct Ctx {
     __device__ __forceinline__ uint8_t *partner_scratch() const {
         return gen + kSmemEpi + (uint32_t)(group * 2 + (colhalf ^ 1)) * (kEpiBytes / 4);
     }
-    // per-column constants of the bt-th B tile this CTA streams (valid from the tile's acc_wait to its release)
-    __device__ __forceinline__ const float4 *extra(int bt) const {
-        return reinterpret_cast<const float4 *>(gen + kSmemExtra + (uint32_t)(bt & (kExtraSlots - 1)) * kExtraBytes);
+    // shared address of the per-column constants of the bt-th B tile this CTA streams (valid from the tile's
+    // extra_wait to its release)
+    __device__ __forceinline__ uint32_t extra(int bt) const {
+        return base + kSmemExtra + (uint32_t)(bt & (kExtraSlots - 1)) * kExtraBytes;
+    }
+    // shared addresses of the scratch of this warp's quad / of its partner quad
+    __device__ __forceinline__ uint32_t epi_addr() const { return base + kSmemEpi + (uint32_t)(group * 2 + colhalf) * (kEpiBytes / 4); }
+    __device__ __forceinline__ uint32_t partner_addr() const {
+        return base + kSmemEpi + (uint32_t)(group * 2 + (colhalf ^ 1)) * (kEpiBytes / 4);
     }
 };
 
