@@ -55,7 +55,7 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // Where everything lives inside the caller's workspace.  One layout serves every entry point.
 struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
-    size_t row_part, cross_part, rn, sort_a, sort_b, mem_tok, mem_w, piece_desc, off, piece_off, part_off, partial;
+    size_t row_part, cross_part, rn, sort_a, sort_b, mem_tok, mem_w, piece_desc, off, piece_off, part_off, partial, ticket;
     size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod, negc;
     int tc_n_qt, tc_n_chunk, tc_tiles_per_chunk, gw_pad;
     size_t total;
@@ -89,6 +89,7 @@ void layout_merge(Layout &y, const flowmm_params &p, Take take) {
     y.piece_off = take(UH * (B + 1) * 4);
     y.part_off = take(UH * (B + 1) * 4);
     y.partial = take(UH * (size_t)y.max_parts * (2 * D + 4) * 4);
+    y.ticket = take(256);
 }
 
 Layout make_layout(const flowmm_params &p) {
@@ -371,7 +372,7 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
     MergeArgs m;
     m.k = k; m.v = v; m.k_out = k_out; m.v_out = v_out; m.retained = retained;
     m.mem_tok = nullptr; m.mem_w = nullptr; m.piece_desc = nullptr; m.piece_off = nullptr; m.part_off = nullptr;
-    m.partial = at<float>(ws, y.partial);
+    m.partial = at<float>(ws, y.partial); m.ticket = nullptr;
     m.Hkv = p.n_kv_heads; m.D = p.head_dim; m.L = p.seq_len; m.B = p.n_keep; m.E = E;
     m.max_pieces = E == 0 ? p.n_keep : y.max_pieces; m.max_parts = y.max_parts;
     for (int i = 0; i < 3; ++i) {
@@ -383,15 +384,16 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
         c.sort_a = at<int>(ws, y.sort_a); c.sort_b = at<int>(ws, y.sort_b);
         c.mem_tok = at<int>(ws, y.mem_tok); c.mem_w = at<float>(ws, y.mem_w);
         c.off = at<int>(ws, y.off); c.piece_off = at<int>(ws, y.piece_off); c.part_off = at<int>(ws, y.part_off);
-        c.piece_desc = at<int4>(ws, y.piece_desc);
+        c.piece_desc = at<int4>(ws, y.piece_desc); c.ticket = at<unsigned>(ws, y.ticket);
         c.B = p.n_keep; c.E = E; c.n_pass = y.csr_passes; c.max_pieces = y.max_pieces; c.merge_mode = p.merge_mode;
         if (E <= 4096) build_csr_kernel<8><<<UH, 256, 0, st>>>(c);
         else build_csr_kernel<32><<<UH, 1024, 0, st>>>(c);
         FLOWMM_LAUNCHED("build_csr");
         m.mem_tok = c.mem_tok; m.mem_w = c.mem_w; m.piece_desc = c.piece_desc;
-        m.piece_off = c.piece_off; m.part_off = c.part_off;
+        m.piece_off = c.piece_off; m.part_off = c.part_off; m.ticket = c.ticket;
     }
     const int64_t total_pieces = (int64_t)UH * m.max_pieces;
+    if (total_pieces > 0xFFFF0000ll) return FLOWMM_ERR_SHAPE;           // the piece table is indexed with 32 bits
     const int64_t want_blocks = (total_pieces + 7) / 8;
     const int gp = (int)(want_blocks < 2 * tc::sm_count() ? want_blocks : 2 * tc::sm_count());   // persistent warps
     const dim3 gf((p.n_keep + 7) / 8, UH);

@@ -109,6 +109,7 @@ struct CsrArgs {
     int *piece_off;          // [UH, B+1] first piece of each slot
     int *part_off;           // [UH, B+1] first partial-sum record of each slot (multi-piece slots only)
     int4 *piece_desc;        // [UH, max_pieces] (slot, first member, members, partial record or -1)
+    unsigned *ticket;        // work counter of the merge kernel, cleared here
     int B, E, n_pass, max_pieces, merge_mode;
 };
 
@@ -122,6 +123,7 @@ __global__ void __launch_bounds__(32 * NW) build_csr_kernel(const CsrArgs A) {
     __shared__ int scratch[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int uh = blockIdx.x;
+    if (uh == 0 && tid == 0) *A.ticket = 0u;
     const int *match = A.match + (int64_t)uh * A.E;
     int *bufs[2] = {A.sort_a + (int64_t)uh * A.E, A.sort_b + (int64_t)uh * A.E};
     const int per_warp = ((A.E + NW - 1) / NW + 31) / 32 * 32;     // multiple of 32
@@ -235,6 +237,7 @@ struct MergeArgs {
     const int4 *piece_desc;           // [UH, max_pieces]
     const int *piece_off, *part_off;  // [UH, B+1]
     float *partial;                   // [UH, max_parts, 2*D + 4] fp32 partial sums
+    unsigned *ticket;                 // shared work counter (pieces are handed out in table order); nullptr: fixed stride
     int Hkv, D, L, B, E, max_pieces, max_parts;
     int64_t ks[3], vs[3], kos[3], vos[3];
 };
@@ -251,21 +254,21 @@ template <typename T>
 __global__ void __launch_bounds__(256) merge_pieces_kernel(const MergeArgs A, int n_uh) {
     constexpr int V = Elem<T>::kVec;
     const int lane = lane_id();
-    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int64_t total = (int64_t)n_uh * A.max_pieces;
+    const unsigned n_warps = gridDim.x * (blockDim.x >> 5);
+    const unsigned total = (unsigned)n_uh * (unsigned)A.max_pieces;
     const int rv = A.D / V;                                   // 16-byte vectors per row
     const int n_vec = 2 * rv;
 
     struct Piece { int4 d; int tok_lo, tok_hi, r; float w_lo, w_hi; };
-    auto fetch_desc = [&](int64_t g) -> int4 {               // (slot, first, count, part); count < 0: no such piece
+    auto fetch_desc = [&](unsigned g) -> int4 {              // (slot, first, count, part); count < 0: no such piece
         if (g >= total) return make_int4(0, 0, -1, -1);
-        if (!A.piece_desc) return make_int4((int)(g % A.max_pieces), 0, 0, -1);      // E == 0: plain copy of the pivots
+        if (!A.piece_desc) return make_int4((int)(g % (unsigned)A.max_pieces), 0, 0, -1);   // E == 0: plain copy of the pivots
         return A.piece_desc[g];
     };
-    auto fetch_members = [&](int64_t g, Piece &pc) {         // needs pc.d
+    auto fetch_members = [&](unsigned g, Piece &pc) {        // needs pc.d
         pc.tok_lo = pc.tok_hi = pc.r = 0; pc.w_lo = pc.w_hi = 0.f;
         if (pc.d.z < 0) return;
-        const int64_t uh = g / A.max_pieces;
+        const int64_t uh = g / (unsigned)A.max_pieces;
         if (pc.d.z > 0) {
             const int *mt = A.mem_tok + uh * A.E + pc.d.y;
             const float *mw = A.mem_w + uh * A.E + pc.d.y;
@@ -274,18 +277,35 @@ __global__ void __launch_bounds__(256) merge_pieces_kernel(const MergeArgs A, in
         }
         if (pc.d.w < 0) pc.r = A.retained[uh * A.B + pc.d.x];
     };
+    // the next piece of this warp: from the shared counter (warps that drew light pieces come back sooner, so
+    // the last pieces end together), or with a fixed stride when there is no counter
+    unsigned stride_next = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    unsigned drawn = 0, drawn_left = 0;                       // pieces are drawn kDraw at a time
+    constexpr unsigned kDraw = 4;
+    auto next_piece = [&]() -> unsigned {
+        if (!A.ticket) { const unsigned g = stride_next; stride_next = g + n_warps < g ? 0xFFFFFFFFu : g + n_warps; return g; }
+        if (drawn_left == 0) {
+            unsigned g = 0;
+            if (lane == 0) g = atomicAdd(A.ticket, kDraw);
+            drawn = __shfl_sync(0xFFFFFFFFu, g, 0);
+            drawn_left = kDraw;
+        }
+        --drawn_left;
+        return drawn++;
+    };
 
-    int64_t g = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    unsigned g = next_piece(), g_nxt = next_piece();
     Piece cur, nxt;
     cur.d = fetch_desc(g);
-    nxt.d = fetch_desc(g + n_warps);
+    nxt.d = fetch_desc(g_nxt);
     fetch_members(g, cur);
-    for (; g < total; g += n_warps) {
-        const int4 d2 = fetch_desc(g + 2 * n_warps);          // two pieces ahead
-        fetch_members(g + n_warps, nxt);                      // one piece ahead
+    while (g < total) {
+        const unsigned g_d2 = next_piece();
+        const int4 d2 = fetch_desc(g_d2);                     // two pieces ahead
+        fetch_members(g_nxt, nxt);                            // one piece ahead
         const int slot = cur.d.x, count = cur.d.z, part = cur.d.w;
         if (count >= 0) {
-            const int uh = (int)(g / A.max_pieces), u = uh / A.Hkv, h = uh % A.Hkv;
+            const int uh = (int)(g / (unsigned)A.max_pieces), u = uh / A.Hkv, h = uh % A.Hkv;
             const T *kb = static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
             const T *vb = static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1];
             for (int vec0 = 0; vec0 < n_vec; vec0 += 32) {    // which vector of the (K row, V row) pair
@@ -348,7 +368,9 @@ __global__ void __launch_bounds__(256) merge_pieces_kernel(const MergeArgs A, in
             }
         }
         cur = nxt;
+        g = g_nxt;
         nxt.d = d2;
+        g_nxt = g_d2;
     }
 }
 
