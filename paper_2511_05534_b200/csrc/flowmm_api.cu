@@ -55,7 +55,7 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // Where everything lives inside the caller's workspace.  One layout serves every entry point.
 struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
-    size_t row_part, cross_part, rn, sort_a, sort_b, mem_tok, mem_w, piece_desc, off, piece_off, part_off, partial, ticket;
+    size_t row_part, cross_part, rn, sort_a, sort_b, mem_tok, mem_w, piece_desc, off, piece_off, part_off, partial, ticket, slot_done;
     size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod, negc;
     int tc_n_qt, tc_n_chunk, tc_tiles_per_chunk, gw_pad;
     size_t total;
@@ -90,6 +90,7 @@ void layout_merge(Layout &y, const flowmm_params &p, Take take) {
     y.part_off = take(UH * (B + 1) * 4);
     y.partial = take(UH * (size_t)y.max_parts * (2 * D + 4) * 4);
     y.ticket = take(256);
+    y.slot_done = take(UH * B * 4);
 }
 
 Layout make_layout(const flowmm_params &p) {
@@ -202,7 +203,7 @@ bool use_tc_score(const flowmm_params &p) {
 }
 
 flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
-                           float *importance, float *cross_mass, void *ws, cudaStream_t st) {
+                           float *importance, float *cross_mass, void *ws, cudaStream_t st, int *parts_out) {
     const int UH = p.n_units * p.n_kv_heads, G = p.n_q_heads / p.n_kv_heads, W = p.window;
     ScoreTcArgs a;
     a.row_part = at<float2>(ws, y.row_part); a.negc = at<float>(ws, y.negc); a.modality = mod;
@@ -238,15 +239,16 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     FLOWMM_LAUNCHED("score_combine");
     score_colsum_tc_kernel<<<a.n_items2 < sms ? a.n_items2 : sms, tcs::kThreads, tcs::kSmemBytes, st>>>(k128, qb, a);
     FLOWMM_LAUNCHED("score_colsum_tc");
+    if (parts_out) { *parts_out = a.n_rt * 8; return FLOWMM_OK; }     // the caller reduces the partial masses itself
     const int n = p.n_units * p.n_q_heads;
-    cross_mass_reduce<<<(n + 255) / 256, 256, 0, st>>>(a.cross_part, a.n_rt * 8, n, cross_mass);
+    cross_mass_reduce<<<(n + 7) / 8, 256, 0, st>>>(a.cross_part, a.n_rt * 8, n, cross_mass);
     FLOWMM_LAUNCHED("cross_mass_reduce");
     return FLOWMM_OK;
 }
 
 flowmm_status run_score(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
-                        float *importance, float *cross_mass, void *ws, cudaStream_t st) {
-    if (use_tc_score(p)) return run_score_tc(p, y, q, k, mod, importance, cross_mass, ws, st);
+                        float *importance, float *cross_mass, void *ws, cudaStream_t st, int *parts_out = nullptr) {
+    if (use_tc_score(p)) return run_score_tc(p, y, q, k, mod, importance, cross_mass, ws, st, parts_out);
     ScoreArgs a;
     a.q = q; a.k = k; a.modality = mod; a.importance = importance;
     a.row_part = at<float2>(ws, y.row_part);
@@ -272,8 +274,9 @@ flowmm_status run_score(const flowmm_params &p, const Layout &y, const void *q, 
         score_colsum_simt<float><<<g2, kSimtThreads, dyn, st>>>(a);
         FLOWMM_LAUNCHED("score_colsum_simt");
     }
+    if (parts_out) { *parts_out = y.n_chunk2; return FLOWMM_OK; }
     const int n = p.n_units * p.n_q_heads;
-    cross_mass_reduce<<<(n + 255) / 256, 256, 0, st>>>(a.cross_part, y.n_chunk2, n, cross_mass);
+    cross_mass_reduce<<<(n + 7) / 8, 256, 0, st>>>(a.cross_part, y.n_chunk2, n, cross_mass);
     FLOWMM_LAUNCHED("cross_mass_reduce");
     return FLOWMM_OK;
 }
@@ -309,8 +312,13 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     g.Hkv = p.n_kv_heads; g.L = p.seq_len; g.B = p.n_keep; g.E = E; g.Ctot = y.c_tot; g.n_rt = y.n_rt;
     g.tau_eff = tau_effective(p);
     for (int i = 0; i < 3; ++i) g.ks[i] = p.k_stride[i];
+    g.copy_here = y.c_tot <= 256;
     match_prepare_kernel<<<UH, 256, 0, st>>>(g);
     FLOWMM_LAUNCHED("match_prepare");
+    if (!g.copy_here) {
+        match_gather_kernel<<<dim3((y.c_tot + 63) / 64, UH), 256, 0, st>>>(g);
+        FLOWMM_LAUNCHED("match_gather");
+    }
 
     CUtensorMap k_map, cand_map;
     const uint64_t kd[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
@@ -372,7 +380,7 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
     MergeArgs m;
     m.k = k; m.v = v; m.k_out = k_out; m.v_out = v_out; m.retained = retained;
     m.mem_tok = nullptr; m.mem_w = nullptr; m.piece_desc = nullptr; m.piece_off = nullptr; m.part_off = nullptr;
-    m.partial = at<float>(ws, y.partial); m.ticket = nullptr;
+    m.partial = at<float>(ws, y.partial); m.ticket = nullptr; m.slot_done = nullptr;
     m.Hkv = p.n_kv_heads; m.D = p.head_dim; m.L = p.seq_len; m.B = p.n_keep; m.E = E;
     m.max_pieces = E == 0 ? p.n_keep : y.max_pieces; m.max_parts = y.max_parts;
     for (int i = 0; i < 3; ++i) {
@@ -384,27 +392,24 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
         c.sort_a = at<int>(ws, y.sort_a); c.sort_b = at<int>(ws, y.sort_b);
         c.mem_tok = at<int>(ws, y.mem_tok); c.mem_w = at<float>(ws, y.mem_w);
         c.off = at<int>(ws, y.off); c.piece_off = at<int>(ws, y.piece_off); c.part_off = at<int>(ws, y.part_off);
-        c.piece_desc = at<int4>(ws, y.piece_desc); c.ticket = at<unsigned>(ws, y.ticket);
+        c.piece_desc = at<int4>(ws, y.piece_desc); c.ticket = at<unsigned>(ws, y.ticket); c.slot_done = at<int>(ws, y.slot_done);
         c.B = p.n_keep; c.E = E; c.n_pass = y.csr_passes; c.max_pieces = y.max_pieces; c.merge_mode = p.merge_mode;
         if (E <= 4096) build_csr_kernel<8><<<UH, 256, 0, st>>>(c);
         else build_csr_kernel<32><<<UH, 1024, 0, st>>>(c);
         FLOWMM_LAUNCHED("build_csr");
         m.mem_tok = c.mem_tok; m.mem_w = c.mem_w; m.piece_desc = c.piece_desc;
-        m.piece_off = c.piece_off; m.part_off = c.part_off; m.ticket = c.ticket;
+        m.piece_off = c.piece_off; m.part_off = c.part_off; m.ticket = c.ticket; m.slot_done = c.slot_done;
     }
     const int64_t total_pieces = (int64_t)UH * m.max_pieces;
     if (total_pieces > 0xFFFF0000ll) return FLOWMM_ERR_SHAPE;           // the piece table is indexed with 32 bits
     const int64_t want_blocks = (total_pieces + 7) / 8;
     const int gp = (int)(want_blocks < 2 * tc::sm_count() ? want_blocks : 2 * tc::sm_count());   // persistent warps
-    const dim3 gf((p.n_keep + 7) / 8, UH);
     if (p.dtype == FLOWMM_BF16) {
         merge_pieces_kernel<__nv_bfloat16><<<gp, 256, 0, st>>>(m, UH);
         FLOWMM_LAUNCHED("merge_pieces");
-        if (E > kPiece) { merge_finish_kernel<__nv_bfloat16><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCHED("merge_finish"); }
     } else {
         merge_pieces_kernel<float><<<gp, 256, 0, st>>>(m, UH);
         FLOWMM_LAUNCHED("merge_pieces");
-        if (E > kPiece) { merge_finish_kernel<float><<<gf, 256, 0, st>>>(m); FLOWMM_LAUNCHED("merge_finish"); }
     }
     return FLOWMM_OK;
 }
@@ -519,8 +524,11 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
     if (!match) match = at<int32_t>(ws, y.match);
     if (!match_sim) match_sim = at<float>(ws, y.match_sim);
     float *cross_mass = at<float>(ws, y.cross_mass);
-    FLOWMM_TRY(run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, st));
-    FLOWMM_TRY(run_layer_flow(*p, cross_mass, rho, strategy, st));
+    int n_parts = 0;
+    FLOWMM_TRY(run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, st, &n_parts));
+    flow_from_parts_kernel<<<p->n_units, 256, 0, st>>>(at<float>(ws, y.cross_part), n_parts, p->n_q_heads, p->window,
+                                                       p->theta, p->flow_mode, cross_mass, rho, strategy);
+    FLOWMM_LAUNCHED("flow_from_parts");
     FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st));
     FLOWMM_TRY(run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws, st));
     FLOWMM_TRY(run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws, st));

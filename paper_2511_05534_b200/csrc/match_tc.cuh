@@ -33,9 +33,36 @@ struct MatchPrepArgs {
     int *rank;                   // [UH, L]  position in the non-pivot list, or -1 for a pivot
     uint8_t *tile_mod;           // [U, n_rt] per tile of 256 tokens; bit 0: holds text tokens, bit 1: visual tokens
     int Hkv, L, B, E, Ctot, n_rt;
+    int copy_here;               // 1: this kernel also gathers the candidate rows; 0: match_gather_kernel does
     float tau_eff;
     int64_t ks[3];
 };
+
+// Copies the candidate key rows (256 bytes each) of positions [lo, hi) of one head's candidate
+// list, 16 lanes per row, and takes each row's reciprocal norm on the way (0 for a zero row: its
+// similarity to anything is 0).  lo, hi multiples of 16; every thread of the block takes part.
+__device__ __forceinline__ void match_gather_rows(const MatchPrepArgs &A, int uh, int lo, int hi, int tid, int nthreads) {
+    const int u = uh / A.Hkv, h = uh % A.Hkv;
+    const int *ret = A.retained + (int64_t)uh * A.B;
+    const int *slot_out = A.cand_slot + (int64_t)uh * A.Ctot;
+    float *scale_out = A.cand_scale + (int64_t)uh * A.Ctot;
+    const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(A.k) + u * A.ks[0] + h * A.ks[1];
+    uint4 *dst = reinterpret_cast<uint4 *>(A.cand_k + (int64_t)uh * A.Ctot * 128);
+    const int sub = tid & 15;
+    for (int pos = lo + (tid >> 4); pos < hi; pos += nthreads >> 4) {       // uniform trip count within a warp
+        const int s = slot_out[pos];
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (s >= 0) val = *reinterpret_cast<const uint4 *>(kb + (int64_t)ret[s] * A.ks[2] + sub * 8);
+        dst[(int64_t)pos * 16 + sub] = val;
+        float x[8], ssq = 0.f;
+        Elem<__nv_bfloat16>::unpack(val, x);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xFFFFFFFFu, ssq, o);
+        if (sub == 0 && s >= 0) scale_out[pos] = ssq > 0.f ? rsqrtf(ssq) : 0.f;
+    }
+}
 
 // grid = U*Hkv, block = 256.
 __global__ void __launch_bounds__(256) match_prepare_kernel(const MatchPrepArgs A) {
@@ -92,24 +119,14 @@ __global__ void __launch_bounds__(256) match_prepare_kernel(const MatchPrepArgs 
     }
     if (tid == 0) { A.cand_count[2 * uh] = seen_t; A.cand_count[2 * uh + 1] = seen_v; }
     __syncthreads();
-    // copy the candidate key rows (256 bytes each), 16 lanes per row, and take each row's reciprocal
-    // norm on the way (0 for a zero row: its similarity to anything is 0)
-    const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(A.k) + u * A.ks[0] + h * A.ks[1];
-    uint4 *dst = reinterpret_cast<uint4 *>(A.cand_k + (int64_t)uh * A.Ctot * 128);
-    const int sub = tid & 15;
-    for (int pos = tid >> 4; pos < A.Ctot; pos += blockDim.x >> 4) {        // Ctot is a multiple of 32: uniform trip count
-        const int s = slot_out[pos];
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (s >= 0) val = *reinterpret_cast<const uint4 *>(kb + (int64_t)ret[s] * A.ks[2] + sub * 8);
-        dst[(int64_t)pos * 16 + sub] = val;
-        float x[8], ssq = 0.f;
-        Elem<__nv_bfloat16>::unpack(val, x);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xFFFFFFFFu, ssq, o);
-        if (sub == 0 && s >= 0) scale_out[pos] = ssq > 0.f ? rsqrtf(ssq) : 0.f;
-    }
+    if (A.copy_here) match_gather_rows(A, uh, 0, A.Ctot, tid, blockDim.x);
+}
+
+// The gather step of the preparation as a kernel of its own for long candidate lists, so that many
+// CTAs share a head's rows.  grid = (ceil(Ctot / 64), U*Hkv), block = 256.
+__global__ void __launch_bounds__(256) match_gather_kernel(const MatchPrepArgs A) {
+    const int lo = blockIdx.x * 64;
+    match_gather_rows(A, blockIdx.y, lo, min(A.Ctot, lo + 64), threadIdx.x, blockDim.x);
 }
 
 struct MatchTcArgs {

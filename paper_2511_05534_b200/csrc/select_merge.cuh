@@ -110,6 +110,7 @@ struct CsrArgs {
     int *part_off;           // [UH, B+1] first partial-sum record of each slot (multi-piece slots only)
     int4 *piece_desc;        // [UH, max_pieces] (slot, first member, members, partial record or -1)
     unsigned *ticket;        // work counter of the merge kernel, cleared here
+    int *slot_done;          // [UH, B] pieces of a slot that have stored their partial sums, cleared here
     int B, E, n_pass, max_pieces, merge_mode;
 };
 
@@ -220,6 +221,7 @@ __global__ void __launch_bounds__(32 * NW) build_csr_kernel(const CsrArgs A) {
         const int pp = piece_seen + block_exclusive_scan(np, scratch, tot_p);
         const int qq = part_seen + block_exclusive_scan(npart, scratch, tot_q);
         if (s <= A.B) { piece_off[s] = pp; part_off[s] = qq; }
+        if (s < A.B) A.slot_done[(int64_t)uh * A.B + s] = 0;
         for (int q = 0; q < np; ++q)
             desc[pp + q] = make_int4(s, off[s] + q * kPiece, min(kPiece, n - q * kPiece), np > 1 ? qq + q : -1);
         piece_seen += tot_p;
@@ -238,9 +240,49 @@ struct MergeArgs {
     const int *piece_off, *part_off;  // [UH, B+1]
     float *partial;                   // [UH, max_parts, 2*D + 4] fp32 partial sums
     unsigned *ticket;                 // shared work counter (pieces are handed out in table order); nullptr: fixed stride
+    int *slot_done;                   // [UH, B] arrival counters of multi-piece slots
     int Hkv, D, L, B, E, max_pieces, max_parts;
     int64_t ks[3], vs[3], kos[3], vos[3];
 };
+
+// A slot whose members were cut into several pieces: add the pieces' partial sums in piece order,
+// then the pivot row, normalise and store.  Run by the warp whose piece was the last to arrive;
+// the partial records come from other SMs, so they are read past L1.
+template <typename T>
+__device__ __forceinline__ void merge_finish_slot(const MergeArgs &A, int uh, int slot, int lane) {
+    constexpr int V = Elem<T>::kVec;
+    const int u = uh / A.Hkv, h = uh % A.Hkv;
+    const int *poff = A.piece_off + (int64_t)uh * (A.B + 1);
+    const int n_pieces = poff[slot + 1] - poff[slot];
+    const int part_base = A.part_off[(int64_t)uh * (A.B + 1) + slot];
+    const float *rec0 = A.partial + ((int64_t)uh * A.max_parts + part_base) * (2 * A.D + 4);
+    const int rv = A.D / V;
+    const int r = A.retained[(int64_t)uh * A.B + slot];
+    float wsum = 0.f;
+    for (int p = 0; p < n_pieces; ++p) wsum += __ldcg(rec0 + (int64_t)p * (2 * A.D + 4) + 2 * A.D);
+    const float inv = 1.f / (1.f + wsum);
+    for (int vec = lane; vec < 2 * rv; vec += 32) {
+        const bool is_v = vec >= rv;
+        const int c0 = (is_v ? vec - rv : vec) * V;
+        float acc[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = 0.f;
+        for (int p = 0; p < n_pieces; ++p) {
+            const float *rec = rec0 + (int64_t)p * (2 * A.D + 4) + (is_v ? A.D : 0) + c0;
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[e] += __ldcg(rec + e);
+        }
+        const T *src = is_v ? static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1] + (int64_t)r * A.vs[2]
+                            : static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1] + (int64_t)r * A.ks[2];
+        T *dst = is_v ? static_cast<T *>(A.v_out) + u * A.vos[0] + h * A.vos[1] + (int64_t)slot * A.vos[2]
+                      : static_cast<T *>(A.k_out) + u * A.kos[0] + h * A.kos[1] + (int64_t)slot * A.kos[2];
+        float x[V], o[V];
+        Elem<T>::load16(src + c0, x);
+#pragma unroll
+        for (int e = 0; e < V; ++e) o[e] = (x[e] + acc[e]) * inv;
+        Elem<T>::store16(dst + c0, o);
+    }
+}
 
 constexpr int kMergeBatch = 8;        // member rows a warp keeps in flight
 
@@ -249,7 +291,8 @@ constexpr int kMergeBatch = 8;        // member rows a warp keeps in flight
 // the current one, so the row loads never wait on index loads.  A 16-byte vector of a K row or V
 // row per lane: with D*sizeof(T) = 256 bytes lanes 0-15 carry the K row and lanes 16-31 the V
 // row.  A single-piece slot is finished here (pivot row with weight 1, Eq. 5 weights, normalise,
-// round once); a piece of a multi-piece slot stores its fp32 partial sums for merge_finish_kernel.
+// round once); a piece of a multi-piece slot stores its fp32 partial sums, and the piece that arrives
+// last adds them up in piece order (so the result does not depend on which piece that was).
 template <typename T>
 __global__ void __launch_bounds__(256) merge_pieces_kernel(const MergeArgs A, int n_uh) {
     constexpr int V = Elem<T>::kVec;
@@ -366,53 +409,23 @@ __global__ void __launch_bounds__(256) merge_pieces_kernel(const MergeArgs A, in
                     if (vec == 0) rec[2 * A.D] = wsum;
                 }
             }
+            if (part >= 0) {                                  // multi-piece slot: was this the last piece to arrive?
+                __threadfence();
+                __syncwarp();
+                int prev = 0;
+                if (lane == 0) prev = atomicAdd(&A.slot_done[(int64_t)uh * A.B + slot], 1);
+                prev = __shfl_sync(0xFFFFFFFFu, prev, 0);
+                const int *poff = A.piece_off + (int64_t)uh * (A.B + 1);
+                if (prev == poff[slot + 1] - poff[slot] - 1) {
+                    __threadfence();
+                    merge_finish_slot<T>(A, uh, slot, lane);
+                }
+            }
         }
         cur = nxt;
         g = g_nxt;
         nxt.d = d2;
         g_nxt = g_d2;
-    }
-}
-
-// Slots whose members were cut into several pieces: add the pieces' partial sums in piece
-// order, then the pivot row, normalise and store.  One warp per slot; grid = (ceil(B/8), U*Hkv).
-template <typename T>
-__global__ void __launch_bounds__(256) merge_finish_kernel(const MergeArgs A) {
-    constexpr int V = Elem<T>::kVec;
-    const int lane = lane_id();
-    const int uh = blockIdx.y, u = uh / A.Hkv, h = uh % A.Hkv;
-    const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (slot >= A.B) return;
-    const int *poff = A.piece_off + (int64_t)uh * (A.B + 1);
-    const int n_pieces = poff[slot + 1] - poff[slot];
-    if (n_pieces <= 1) return;
-    const int part_base = A.part_off[(int64_t)uh * (A.B + 1) + slot];
-    const float *rec0 = A.partial + ((int64_t)uh * A.max_parts + part_base) * (2 * A.D + 4);
-    const int rv = A.D / V;
-    const int r = A.retained[(int64_t)uh * A.B + slot];
-    float wsum = 0.f;
-    for (int p = 0; p < n_pieces; ++p) wsum += rec0[(int64_t)p * (2 * A.D + 4) + 2 * A.D];
-    const float inv = 1.f / (1.f + wsum);
-    for (int vec = lane; vec < 2 * rv; vec += 32) {
-        const bool is_v = vec >= rv;
-        const int c0 = (is_v ? vec - rv : vec) * V;
-        float acc[V];
-#pragma unroll
-        for (int e = 0; e < V; ++e) acc[e] = 0.f;
-        for (int p = 0; p < n_pieces; ++p) {
-            const float *rec = rec0 + (int64_t)p * (2 * A.D + 4) + (is_v ? A.D : 0) + c0;
-#pragma unroll
-            for (int e = 0; e < V; ++e) acc[e] += rec[e];
-        }
-        const T *src = is_v ? static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1] + (int64_t)r * A.vs[2]
-                            : static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1] + (int64_t)r * A.ks[2];
-        T *dst = is_v ? static_cast<T *>(A.v_out) + u * A.vos[0] + h * A.vos[1] + (int64_t)slot * A.vos[2]
-                      : static_cast<T *>(A.k_out) + u * A.kos[0] + h * A.kos[1] + (int64_t)slot * A.kos[2];
-        float x[V], o[V];
-        Elem<T>::load16(src + c0, x);
-#pragma unroll
-        for (int e = 0; e < V; ++e) o[e] = (x[e] + acc[e]) * inv;
-        Elem<T>::store16(dst + c0, o);
     }
 }
 
