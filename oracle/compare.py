@@ -157,7 +157,9 @@ def compare(p: O.OracleParams, q, k, v, modality, g: Dict[str, np.ndarray], bf16
         stats["match_sim_max_abs"] = float(serr.max(initial=0))
     stats["match_near_ties"] = n_match_ties
     if row_step != 1:
-        return stats
+        # only every row_step-th non-pivot was matched by the oracle: the rows in between carry the
+        # other side's similarity (the sampled ones have just been validated), the merge itself is exact
+        sim_forced = np.where(evaluated, sim_forced, g["match_sim"]) if E > 0 else sim_forced
 
     ko, vo, _ = O.merge(p, k, v, forced["retained"], forced["evicted"], g["match"], sim_forced)
     for name, ref in (("k_out", ko), ("v_out", vo)):
