@@ -196,9 +196,6 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             const int token = p.rt * kMtItemRows + c.group * kMtRows + row;
             const bool in_range = token < A.L;
             const int my_mod = in_range ? A.modality[(int64_t)p.u * A.L + token] : 0;
-            // admissible columns of this row; only consulted where rows of a tile differ (row_masked)
-            int r1hi = p.n_text, r2lo = p.t0, r2hi = p.t0 + p.n_vis;
-            if (p.intra) { if (my_mod == 0) r2hi = r2lo; else r1hi = 0; }
             const bool row_masked = p.intra && p.mixed;
             float best = -INFINITY;
             int best_cc = -1;
@@ -232,29 +229,32 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
                     if (!ok) break;
                     const uint32_t scale4 = c.extra(bt);             // reciprocal norms of this tile's candidates
-                    // one chunk of 32 columns; kMasked: rows of the tile differ in which columns they may take
-                    auto chunk = [&](auto masked_tag, int ch, uint32_t (&acc)[32]) {
+                    // one block of 16 columns; kMasked: rows of the tile differ in which columns they may take
+                    auto block = [&](auto masked_tag, int blk, uint32_t (&acc)[16]) {
                         constexpr bool kMasked = decltype(masked_tag)::value;
-                        const int cc = col0 + ch * 32;
-                        float v[32];
+                        const int cc = col0 + blk * 16;
+                        float v[16];
 #pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4) {     // a column that is no candidate has scale NaN and never wins
-                            const float4 s4 = tc::lds128(scale4 + (ch * 8 + q4) * 16);
+                        for (int q4 = 0; q4 < 4; ++q4) {     // a column that is no candidate has scale NaN and never wins
+                            const float4 s4 = tc::lds128(scale4 + (blk * 4 + q4) * 16);
                             v[4 * q4 + 0] = __uint_as_float(acc[4 * q4 + 0]) * s4.x;
                             v[4 * q4 + 1] = __uint_as_float(acc[4 * q4 + 1]) * s4.y;
                             v[4 * q4 + 2] = __uint_as_float(acc[4 * q4 + 2]) * s4.z;
                             v[4 * q4 + 3] = __uint_as_float(acc[4 * q4 + 3]) * s4.w;
                         }
                         if constexpr (kMasked) {             // intra-modal layer, tile with tokens of both modalities
+                            // admissible columns of this row
+                            int r1hi = p.n_text, r2lo = p.t0, r2hi = p.t0 + p.n_vis;
+                            if (my_mod == 0) r2hi = r2lo; else r1hi = 0;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
+                            for (int j = 0; j < 16; ++j) {
                                 const int col = cc + j;
                                 const bool valid = (col < r1hi) || (col >= r2lo && col < r2hi);
                                 v[j] = valid ? v[j] : -INFINITY;
                             }
                         }
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) {        // four groups of 8 columns, in column order
+                        for (int g = 0; g < 2; ++g) {        // two groups of 8 columns, in column order
                             const float q8 = tc::max3(tc::max3(v[8 * g], v[8 * g + 1], v[8 * g + 2]),
                                                       tc::max3(v[8 * g + 3], v[8 * g + 4], v[8 * g + 5]),
                                                       fmaxf(v[8 * g + 6], v[8 * g + 7]));
@@ -267,11 +267,11 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                             }
                         }
                     };
-                    const int n_chunks = (ncols + 31) >> 5;
+                    const int n_blocks = (ncols + 15) >> 4;
                     if (row_masked)
-                        tcs::for_each_chunk(c, n_chunks, [&](int ch, uint32_t (&acc)[32]) { chunk(std::true_type{}, ch, acc); });
+                        tcs::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::true_type{}, blk, acc); });
                     else
-                        tcs::for_each_chunk(c, n_chunks, [&](int ch, uint32_t (&acc)[32]) { chunk(std::false_type{}, ch, acc); });
+                        tcs::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::false_type{}, blk, acc); });
                     tcs::acc_release(c);
                 }
             }

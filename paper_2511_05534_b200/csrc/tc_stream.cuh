@@ -251,6 +251,18 @@ __device__ __forceinline__ void for_each_chunk(const Ctx &c, int n_chunks, F &&f
         f(ch, a);
     }
 }
+// The same walk in blocks of 16 columns (for epilogues that are short of registers): f(block, values)
+// for blocks 8*colhalf .. 8*colhalf+7 below n_blocks = ceil(columns of the tile / 16).
+template <class F>
+__device__ __forceinline__ void for_each_block16(const Ctx &c, int n_blocks, F &&f) {
+    const int hi = min(n_blocks, 8 * c.colhalf + 8);
+    for (int b = 8 * c.colhalf; b < hi; ++b) {
+        uint32_t a[16];
+        tc::tmem_ld16(c.tmem_base + c.group * kCols + b * 16 + ((uint32_t)(c.quarter * 32) << 16), a);
+        tc::tmem_ld_wait(a);
+        f(b, a);
+    }
+}
 // Meeting point of the two warps that share rows (same half, same lanes, other columns).
 __device__ __forceinline__ void pair_sync(const Ctx &c) {
     asm volatile("bar.sync %0, 64;" ::"r"(1 + c.group * 4 + c.quarter) : "memory");
