@@ -107,7 +107,7 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
                                 add0 += tc::ex2(fmaf(raw[j], A.scale_log2, neg));
                                 add1 += tc::ex2(fmaf(raw[j + 1], A.scale_log2, neg));
                                 add2 += tc::ex2(fmaf(raw[j + 2], A.scale_log2, neg));
-                                add3 += tc::ex2(fmaf(raw[j + 3], A.scale_log2, neg));
+                                add3 += tc::ex2_fma(fmaf(raw[j + 3], A.scale_log2, neg));     // every fourth one on the FMA pipe
                             }
                         } else {
                             float s[32];

@@ -209,6 +209,24 @@ __device__ __forceinline__ float ex2(float x) {        // 2^x, hardware approxim
     return y;
 }
 
+// 2^x on the FMA pipe (relative error 2.2e-7 for x in [-125, 127]; smaller x give 2^-125): round x to
+// the nearest integer n with the 1.5 * 2^23 trick, a degree-5 polynomial for 2^f on f = x - n in
+// [-0.5, 0.5] (own least-squares fit at Chebyshev nodes), then n is added to the exponent field.
+// The exp2 unit does 16 results per clock per SM; the row-statistics pass of the scoring step, which
+// is bound by that unit, sends a quarter of its exponentials here.
+__device__ __forceinline__ float ex2_fma(float x) {
+    x = fmaxf(x, -125.f);
+    const float t = x + 12582912.f;
+    const float f = x - (t - 12582912.f);
+    float p = 0.0013266971f;
+    p = fmaf(p, f, 0.0096754599f);
+    p = fmaf(p, f, 0.055507425f);
+    p = fmaf(p, f, 0.24022122f);
+    p = fmaf(p, f, 0.69314694f);
+    p = fmaf(p, f, 1.0000001f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float m;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
