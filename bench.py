@@ -147,6 +147,13 @@ def kernel_model(wl, B, dsize):
     return m
 
 
+# DRAM bytes (read + write) of one launch from `ncu --set full` captures of the committed kernels on
+# the whole stack of the workload (profiles/ has the commands); None where no capture was taken.
+NCU_TRAFFIC = {
+    ("cfg2", 100): {"merge_pieces": 377.3e6, "match_tc": 202.7e6},
+    ("cfg4", 200): {"match_tc": 305.3e6, "score_stats_tc": 260.2e6, "score_colsum_tc": 262.1e6, "merge_pieces": 580.4e6},
+}
+
 KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
     "score_stats_simt": "score_stats", "score_stats_tc": "score_stats",
     "score_colsum_simt": "score_colsum", "score_colsum_tc": "score_colsum",
@@ -340,6 +347,10 @@ def run_ours(args):
         roofline = {"kernel": top, "bound": "hbm", "achieved": tk["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": tk["frac"], "traffic": None, "peak_source": peaks["source"]}
     roofline["launch_ms"] = tk["ms"]
+    if n_layers == wl.n_layers:
+        roofline["traffic"] = NCU_TRAFFIC.get((wl.name, args.permille), {}).get(top)
+    roofline["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)"
+    roofline["algorithmic_bytes"] = model_for(top, model)[1] * U
 
     # end to end: pinned host inputs -> device -> compress -> pinned host result, every step
     hq, hk, hv, hm = (t.cpu().pin_memory() for t in sets[0])
