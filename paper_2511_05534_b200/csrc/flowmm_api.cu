@@ -115,7 +115,7 @@ Layout make_layout(const flowmm_params &p) {
     {   // pass 1 of the tensor-core scoring: key chunks of whole 256-key tiles, sized so that the
         // persistent CTAs (one per SM, 148 on B200) finish their last round together
         y.tc_n_qt = (int)((G * W + tcs::kItemRows - 1) / tcs::kItemRows);
-        const int key_tiles = (int)((L + tcs::kCols - 1) / tcs::kCols);
+        const int key_tiles = (int)((L + tcs::Big::kCols - 1) / tcs::Big::kCols);
         const long base_items = (long)(U * Hkv) * y.tc_n_qt;
         double best_cost = 1e300;
         y.tc_tiles_per_chunk = key_tiles;
@@ -127,7 +127,7 @@ Layout make_layout(const flowmm_params &p) {
             if (cost < best_cost - 1e-9) { best_cost = cost; y.tc_tiles_per_chunk = tpc; }
         }
         y.tc_n_chunk = (key_tiles + y.tc_tiles_per_chunk - 1) / y.tc_tiles_per_chunk;
-        y.gw_pad = (int)((G * W + tcs::kCols - 1) / tcs::kCols * tcs::kCols);
+        y.gw_pad = (int)((G * W + tcs::Big::kCols - 1) / tcs::Big::kCols * tcs::Big::kCols);
     }
     const size_t max_chunk1 = (size_t)(y.n_chunk1 > 2 * y.tc_n_chunk ? y.n_chunk1 : 2 * y.tc_n_chunk);
     const size_t max_chunk2 = (size_t)(y.n_chunk2 > 8 * y.n_rt ? y.n_chunk2 : 8 * y.n_rt);
@@ -211,7 +211,11 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.G = G; a.W = W; a.L = p.seq_len; a.GW = G * W; a.GWpad = y.gw_pad;
     a.n_qt = y.tc_n_qt; a.n_chunk = y.tc_n_chunk; a.tiles_per_chunk = y.tc_tiles_per_chunk; a.n_rt = y.n_rt;
     a.a_heads = G < tcs::kRows / W ? G : tcs::kRows / W;        // one A half holds 128 proxy rows
-    a.b_heads = G < tcs::kCols / W ? G : tcs::kCols / W;
+    // pass 2 streams the keys as the A operand; with few proxy rows per KV head the small shape (two A stages)
+    // keeps the key loads in flight across items
+    const bool small2 = a.GW <= 128 && W <= 64;
+    const int nb2 = small2 ? tcs::Small::kCols : tcs::Big::kCols;
+    a.b_heads = G < nb2 / W ? G : nb2 / W;
     a.n_items1 = UH * a.n_qt * a.n_chunk; a.n_items2 = UH * a.n_rt;
     const float scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * kLog2e;
@@ -222,22 +226,27 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     const uint64_t kd[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
     const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
     const uint32_t bqa[4] = {64, (uint32_t)W, (uint32_t)a.a_heads, 1}, bqb[4] = {64, (uint32_t)W, (uint32_t)a.b_heads, 1};
-    const uint32_t bk128[4] = {64, tcs::kRows, 1, 1}, bk256[4] = {64, tcs::kCols, 1, 1};
+    const uint32_t bk128[4] = {64, tcs::kRows, 1, 1}, bk256[4] = {64, tcs::Big::kCols, 1, 1};
     if (!tc::make_bf16_map(&qa, q, 4, qd, qs, bqa) || !tc::make_bf16_map(&qb, q, 4, qd, qs, bqb) ||
         !tc::make_bf16_map(&k128, k, 4, kd, ks, bk128) || !tc::make_bf16_map(&k256, k, 4, kd, ks, bk256))
         return FLOWMM_ERR_CUDA;
-    if (cudaFuncSetAttribute(score_stats_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)tcs::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(score_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)tcs::kSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(score_stats_tc_kernel<tcs::Big>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::Big::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(score_colsum_tc_kernel<tcs::Big>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::Big::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(score_colsum_tc_kernel<tcs::Small>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::Small::kSmemBytes) != cudaSuccess)
         return FLOWMM_ERR_CUDA;
     const int sms = tc::sm_count();
-    score_stats_tc_kernel<<<a.n_items1 < sms ? a.n_items1 : sms, tcs::kThreads, tcs::kSmemBytes, st>>>(qa, k256, a);
+    score_stats_tc_kernel<tcs::Big><<<a.n_items1 < sms ? a.n_items1 : sms, tcs::kThreads, tcs::Big::kSmemBytes, st>>>(qa, k256, a);
     FLOWMM_LAUNCHED("score_stats_tc");
     const int n_negc = UH * a.GWpad;
     score_combine_kernel<<<(n_negc + 255) / 256, 256, 0, st>>>(a.row_part, 2 * a.n_chunk, a.GW, a.GWpad, UH, a.negc);
     FLOWMM_LAUNCHED("score_combine");
-    score_colsum_tc_kernel<<<a.n_items2 < sms ? a.n_items2 : sms, tcs::kThreads, tcs::kSmemBytes, st>>>(k128, qb, a);
+    if (small2)
+        score_colsum_tc_kernel<tcs::Small><<<a.n_items2 < sms ? a.n_items2 : sms, tcs::kThreads, tcs::Small::kSmemBytes, st>>>(k128, qb, a);
+    else
+        score_colsum_tc_kernel<tcs::Big><<<a.n_items2 < sms ? a.n_items2 : sms, tcs::kThreads, tcs::Big::kSmemBytes, st>>>(k128, qb, a);
     FLOWMM_LAUNCHED("score_colsum_tc");
     if (parts_out) { *parts_out = a.n_rt * 8; return FLOWMM_OK; }     // the caller reduces the partial masses itself
     const int n = p.n_units * p.n_q_heads;
@@ -325,7 +334,10 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
     const uint64_t cd[4] = {128, (uint64_t)y.c_tot, (uint64_t)UH, 1};
     const uint64_t cs[3] = {256, (uint64_t)y.c_tot * 256, (uint64_t)y.c_tot * 256 * (uint64_t)UH};
-    const uint32_t box_a[4] = {64, kMtRows, 1, 1}, box_b[4] = {64, kMtCols, 1, 1};
+    // few candidates per head: the token rows are the stream, take the shape with two A stages
+    const bool small = y.c_tot <= 128;
+    const uint32_t box_a[4] = {64, kMtRows, 1, 1};
+    const uint32_t box_b[4] = {64, (uint32_t)(small ? tcs::Small::kCols : tcs::Big::kCols), 1, 1};
     if (!tc::make_bf16_map(&k_map, k, 4, kd, ks, box_a) || !tc::make_bf16_map(&cand_map, g.cand_k, 4, cd, cs, box_b))
         return FLOWMM_ERR_CUDA;
     MatchTcArgs a;
@@ -333,11 +345,14 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     a.cand_scale = g.cand_scale; a.modality = mod; a.tile_mod = g.tile_mod;
     a.match = match; a.match_sim = match_sim; a.status = at<int>(ws, y.status);
     a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.E = E; a.Ctot = y.c_tot; a.n_rt = y.n_rt; a.n_items = UH * y.n_rt;
-    if (cudaFuncSetAttribute(match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tcs::kSmemBytes) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(match_tc_kernel<tcs::Big>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::Big::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(match_tc_kernel<tcs::Small>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::Small::kSmemBytes) != cudaSuccess)
         return FLOWMM_ERR_CUDA;
     const int grid = a.n_items < tc::sm_count() ? a.n_items : tc::sm_count();
-    match_tc_kernel<<<grid, tcs::kThreads, tcs::kSmemBytes, st>>>(k_map, cand_map, a);
+    if (small) match_tc_kernel<tcs::Small><<<grid, tcs::kThreads, tcs::Small::kSmemBytes, st>>>(k_map, cand_map, a);
+    else match_tc_kernel<tcs::Big><<<grid, tcs::kThreads, tcs::Big::kSmemBytes, st>>>(k_map, cand_map, a);
     FLOWMM_LAUNCHED("match_tc");
     return FLOWMM_OK;
 }

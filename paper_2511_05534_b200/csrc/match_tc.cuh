@@ -19,7 +19,6 @@ namespace flowmm {
 
 constexpr int kMtRows = tcs::kRows;          // tokens per accumulator half
 constexpr int kMtItemRows = tcs::kItemRows;  // tokens per item (two halves)
-constexpr int kMtCols = tcs::kCols;          // candidates per column tile
 
 struct MatchPrepArgs {
     const void *k;
@@ -145,16 +144,32 @@ struct MatchItem {
     tcs::TilePlan tp;
 };
 
+// What an item's plan reads from global memory; kept apart so that a role can fetch the next item's
+// values while it works on the current one.
+struct MatchRaw { int n_text, n_vis, strategy, tile_mod; };
+
+__device__ __forceinline__ MatchRaw match_raw(const MatchTcArgs &A, int item) {
+    MatchRaw r = {0, 0, 1, 0};
+    if (item >= A.n_items) return r;
+    const int uh = item / A.n_rt, rt = item % A.n_rt, u = uh / A.Hkv;
+    r.n_text = A.cand_count[2 * uh]; r.n_vis = A.cand_count[2 * uh + 1];
+    r.strategy = A.strategy[u];
+    r.tile_mod = A.tile_mod[(int64_t)u * A.n_rt + rt];
+    return r;
+}
+
 // Which candidate columns a tile of 256 tokens has to visit: everything in a cross-modal layer or
 // when the tile mixes modalities, otherwise only the group of the tile's modality.
-__device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) {
+template <class S>
+__device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item, const MatchRaw &raw) {
+    constexpr int kMtCols = S::kCols;        // candidates per column tile
     MatchItem p;
     p.uh = item / A.n_rt; p.rt = item % A.n_rt;
     p.u = p.uh / A.Hkv; p.h = p.uh % A.Hkv;
-    p.n_text = A.cand_count[2 * p.uh]; p.n_vis = A.cand_count[2 * p.uh + 1];
+    p.n_text = raw.n_text; p.n_vis = raw.n_vis;
     p.t0 = (p.n_text + 31) & ~31;
-    p.intra = A.strategy[p.u] == 0;
-    const int tm = A.tile_mod[(int64_t)p.u * A.n_rt + p.rt];
+    p.intra = raw.strategy == 0;
+    const int tm = raw.tile_mod;
     p.mixed = tm == 3;
     const int end_all = p.n_vis > 0 ? p.t0 + p.n_vis : p.n_text;
     if (!p.intra || tm == 3) { p.lo = 0; p.hi = end_all; }
@@ -171,31 +186,54 @@ __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) 
     p.tp.extra = A.cand_scale + (int64_t)p.uh * A.Ctot + p.lo;
     return p;
 }
+template <class S>
+__device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) {
+    return match_plan<S>(A, item, match_raw(A, item));
+}
 
 // Persistent kernel, one CTA per SM; item = (unit, head, tile of 256 tokens).
+template <class S>
 __global__ void __launch_bounds__(tcs::kThreads, 1)
 match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap cand_map,
                 const MatchTcArgs A) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &cand_map, A.status, 4);
+    constexpr int kMtCols = S::kCols;
+    const typename S::Ctx c = S::setup(smem_raw, &k_map, &cand_map, A.status, 4);
     if (!c.ok) return;
-    auto plan = [&](int item) { return match_plan(A, item).tp; };
+    auto plan = [&](int item) { return match_plan<S>(A, item).tp; };
     if (c.warp == 0) {
-        if (c.lane == 0) tcs::producer(c, &k_map, &cand_map, A.n_items, tcs::kAHalf, tcs::kBStage, plan, A.status);
+        if (c.lane == 0) S::producer(c, &k_map, &cand_map, A.n_items, tcs::kAHalf, S::kBStage, plan, A.status);
     } else if (c.warp == 1) {
-        if (c.lane == 0) tcs::mma_issuer(c, A.n_items, plan, A.status);
+        if (c.lane == 0) S::mma_issuer(c, A.n_items, plan, A.status);
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
         const uint32_t wrow = c.epi_addr() + row * 32;          // 8 floats per row
         const uint32_t prow = c.partner_addr() + row * 32;      // the other column half's
         int k = 0, bt = 0, n_mine = 0;
         bool ok = true;
+        // what an item needs from global memory is fetched one item ahead: its plan values, the token's
+        // modality and its place in the non-pivot list
+        auto token_of = [&](int item) { return (item % A.n_rt) * kMtItemRows + c.group * kMtRows + row; };
+        auto fetch_mod = [&](int item) -> int {
+            const int token = token_of(item);
+            return item < A.n_items && token < A.L ? A.modality[(int64_t)(item / A.n_rt / A.Hkv) * A.L + token] : 0;
+        };
+        auto fetch_rank = [&](int item) -> int {
+            const int token = token_of(item);
+            return item < A.n_items && token < A.L ? A.rank[(int64_t)(item / A.n_rt) * A.L + token] : -1;
+        };
+        MatchRaw raw_next = match_raw(A, blockIdx.x);
+        int mod_next = fetch_mod(blockIdx.x), rank_next = fetch_rank(blockIdx.x);
         for (int item = blockIdx.x; ok && item < A.n_items; item += gridDim.x) {
-            const MatchItem p = match_plan(A, item);
+            const MatchRaw raw = raw_next;
+            const int my_mod = mod_next, my_rank = rank_next;
+            raw_next = match_raw(A, item + gridDim.x);
+            mod_next = fetch_mod(item + gridDim.x);
+            rank_next = fetch_rank(item + gridDim.x);
+            const MatchItem p = match_plan<S>(A, item, raw);
             const bool active = !p.tp.empty() && c.group < p.tp.n_halves;
             const int token = p.rt * kMtItemRows + c.group * kMtRows + row;
             const bool in_range = token < A.L;
-            const int my_mod = in_range ? A.modality[(int64_t)p.u * A.L + token] : 0;
             const bool row_masked = p.intra && p.mixed;
             float best = -INFINITY;
             int best_cc = -1;
@@ -206,8 +244,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 if (c.colhalf == 0) {
                     // the token's key row sits in this half's A stage (128-byte rows, 16-byte units XOR-swizzled by
                     // the row index): read it once for the norm while the first MMAs run, then hand the stage back
-                    ok = tcs::a_wait(c, n_mine++, A.status);
-                    const uint32_t a_half = c.base + tcs::kSmemA + c.group * tcs::kAHalf + row * 128;
+                    ok = S::a_wait(c, n_mine, A.status);
+                    const uint32_t a_half = c.a_addr(n_mine) + row * 128;
 #pragma unroll
                     for (int kh = 0; kh < 2; ++kh) {
 #pragma unroll
@@ -221,12 +259,12 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                             for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
                         }
                     }
-                    tcs::a_release(c);
+                    S::a_release(c, n_mine++);
                 }
                 for (int t = 0; ok && t < p.tp.n_tiles; ++t, ++k, ++bt) {
                     const int col0 = p.lo + t * kMtCols;
                     const int ncols = min(kMtCols, p.hi - col0);
-                    ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
+                    ok = S::extra_wait(c, bt, A.status) && S::acc_wait(c, k, A.status);
                     if (!ok) break;
                     const uint32_t scale4 = c.extra(bt);             // reciprocal norms of this tile's candidates
                     // one block of 16 columns; kMasked: rows of the tile differ in which columns they may take
@@ -269,10 +307,10 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     };
                     const int n_blocks = (ncols + 15) >> 4;
                     if (row_masked)
-                        tcs::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::true_type{}, blk, acc); });
+                        S::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::true_type{}, blk, acc); });
                     else
-                        tcs::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::false_type{}, blk, acc); });
-                    tcs::acc_release(c);
+                        S::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::false_type{}, blk, acc); });
+                    S::acc_release(c);
                 }
             }
             // (after a wait that ran out the results are garbage, but the two meeting points below are still
@@ -293,12 +331,12 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             }
             // the upper column half hands its result to the lower one, which owns the row's output
             if (c.colhalf == 1) tc::sts128(wrow, best, __int_as_float(slot), 0.f, 0.f);
-            tcs::pair_sync(c);
+            S::pair_sync(c);
             if (c.colhalf == 0 && ok) {
                 const float4 other = tc::lds128(prow);
                 if (other.x > best) { best = other.x; slot = __float_as_int(other.y); }    // a tie stays with the lower columns
                 if (in_range) {
-                    const int j = A.rank[(int64_t)p.uh * A.L + token];
+                    const int j = my_rank;
                     if (j >= 0) {                                    // a non-pivot: report its match
                         float sim = 0.f;
                         if (slot >= 0 && ssq > 0.f) sim = best * rsqrtf(ssq);
@@ -307,10 +345,10 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     }
                 }
             }
-            tcs::pair_sync(c);                                       // the hand-over slot may be overwritten again
+            S::pair_sync(c);                                       // the hand-over slot may be overwritten again
         }
     }
-    tcs::teardown(c);
+    S::teardown(c);
 }
 
 }  // namespace flowmm

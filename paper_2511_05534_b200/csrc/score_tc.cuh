@@ -47,32 +47,33 @@ __device__ __forceinline__ float max32(const float (&v)[32]) {
 
 // ---------------------------------------------------------------------------------------------
 // Pass 1.  item = (unit*head, tile of 256 proxy rows, key chunk).
+template <class S>
 __global__ void __launch_bounds__(tcs::kThreads, 1)
 score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                       const ScoreTcArgs A) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const tcs::Ctx c = tcs::setup(smem_raw, &q_map, &k_map, A.status);
+    const typename S::Ctx c = S::setup(smem_raw, &q_map, &k_map, A.status);
     if (!c.ok) return;
     auto plan = [&](int item) {
         tcs::TilePlan p;
         const int kc = item % A.n_chunk, qt = (item / A.n_chunk) % A.n_qt, uh = item / (A.n_chunk * A.n_qt);
         const int u = uh / A.Hkv, h = uh % A.Hkv;
-        const int key0 = kc * A.tiles_per_chunk * tcs::kCols;
-        const int keys = min(A.L - key0, A.tiles_per_chunk * tcs::kCols);
+        const int key0 = kc * A.tiles_per_chunk * S::kCols;
+        const int keys = min(A.L - key0, A.tiles_per_chunk * S::kCols);
         p.a1 = 0; p.a2 = h * A.G + qt * (tcs::kItemRows / A.W); p.a3 = u;
         p.h1 = 0; p.h2 = tcs::kRows / A.W;
         p.n_halves = qt * tcs::kItemRows + tcs::kRows < A.GW ? 2 : 1;
-        p.b1 = key0; p.b2 = h; p.b3 = u; p.step1 = tcs::kCols; p.step2 = 0;
+        p.b1 = key0; p.b2 = h; p.b3 = u; p.step1 = S::kCols; p.step2 = 0;
         p.cols_total = keys > 0 ? keys : 0;
-        p.n_tiles = (p.cols_total + tcs::kCols - 1) / tcs::kCols;
+        p.n_tiles = (p.cols_total + S::kCols - 1) / S::kCols;
         p.extra = nullptr;
         return p;
     };
     const uint32_t a_bytes = (uint32_t)A.a_heads * A.W * 256u;
     if (c.warp == 0) {
-        if (c.lane == 0) tcs::producer(c, &q_map, &k_map, A.n_items1, a_bytes, tcs::kBStage, plan, A.status);
+        if (c.lane == 0) S::producer(c, &q_map, &k_map, A.n_items1, a_bytes, S::kBStage, plan, A.status);
     } else if (c.warp == 1) {
-        if (c.lane == 0) tcs::mma_issuer(c, A.n_items1, plan, A.status);
+        if (c.lane == 0) S::mma_issuer(c, A.n_items1, plan, A.status);
     } else {
         const int row_in_half = c.quarter * 32 + c.lane;
         int k = 0;
@@ -87,12 +88,12 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
             const int pa = A.L - A.W + (r % A.W);                    // last key this proxy row may see
             float m = kNegBig, l = 0.f;
             for (int t = 0; ok && t < p.n_tiles; ++t, ++k) {
-                ok = tcs::acc_wait(c, k, A.status);
+                ok = S::acc_wait(c, k, A.status);
                 if (!ok) break;
-                const int kb = p.b1 + t * tcs::kCols;
-                const int ncols = min(tcs::kCols, p.cols_total - t * tcs::kCols);
+                const int kb = p.b1 + t * S::kCols;
+                const int ncols = min(S::kCols, p.cols_total - t * S::kCols);
                 if (warp_has_rows) {
-                    tcs::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
+                    S::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
                         const int k0 = kb + ch * 32;
                         float mx;
                         float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
@@ -129,13 +130,13 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
                         m = mx;
                     });
                 }
-                tcs::acc_release(c);
+                S::acc_release(c);
             }
             if (!ok) break;
             if (valid_row) A.row_part[((int64_t)uh * A.GW + r) * (2 * A.n_chunk) + 2 * kc + c.colhalf] = make_float2(m, l);
         }
     }
-    tcs::teardown(c);
+    S::teardown(c);
 }
 
 // Row constants for pass 2: negc[r] = -(M_r + log2 Z_r) so that exp2(s + negc) is the softmax
@@ -158,11 +159,12 @@ __global__ void score_combine_kernel(const float2 *row_part, int n_chunk, int GW
 
 // ---------------------------------------------------------------------------------------------
 // Pass 2.  item = (unit*head, tile of 256 keys); the B stream is the head group's proxy rows.
+template <class S>
 __global__ void __launch_bounds__(tcs::kThreads, 1)
 score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap q_map,
                        const ScoreTcArgs A) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const tcs::Ctx c = tcs::setup(smem_raw, &k_map, &q_map, A.status);
+    const typename S::Ctx c = S::setup(smem_raw, &k_map, &q_map, A.status);
     if (!c.ok) return;
     auto plan = [&](int item) {
         tcs::TilePlan p;
@@ -171,17 +173,17 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
         p.a1 = kt * tcs::kItemRows; p.a2 = h; p.a3 = u;
         p.h1 = tcs::kRows; p.h2 = 0;
         p.n_halves = p.a1 + tcs::kRows < A.L ? 2 : 1;
-        p.b1 = 0; p.b2 = h * A.G; p.b3 = u; p.step1 = 0; p.step2 = tcs::kCols / A.W;
+        p.b1 = 0; p.b2 = h * A.G; p.b3 = u; p.step1 = 0; p.step2 = S::kCols / A.W;
         p.cols_total = A.GW;
-        p.n_tiles = (A.GW + tcs::kCols - 1) / tcs::kCols;
+        p.n_tiles = (A.GW + S::kCols - 1) / S::kCols;
         p.extra = A.negc + (int64_t)uh * A.GWpad;        // row constants of pass 1, 256 per B tile
         return p;
     };
     const uint32_t b_bytes = (uint32_t)A.b_heads * A.W * 256u;
     if (c.warp == 0) {
-        if (c.lane == 0) tcs::producer(c, &k_map, &q_map, A.n_items2, tcs::kAHalf, b_bytes, plan, A.status);
+        if (c.lane == 0) S::producer(c, &k_map, &q_map, A.n_items2, tcs::kAHalf, b_bytes, plan, A.status);
     } else if (c.warp == 1) {
-        if (c.lane == 0) tcs::mma_issuer(c, A.n_items2, plan, A.status);
+        if (c.lane == 0) S::mma_issuer(c, A.n_items2, plan, A.status);
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
         const uint32_t xch = c.epi_addr() + row * 4;            // hand-over slot of this row
@@ -216,12 +218,12 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
             float imp = 0.f, cg = 0.f;
             int cur_g = -1;                                          // head whose mass is being summed; -1: none yet
             for (int t = 0; ok && t < p.n_tiles; ++t, ++k, ++bt) {
-                const int ncols = min(tcs::kCols, A.GW - t * tcs::kCols);
-                ok = tcs::extra_wait(c, bt, A.status) && tcs::acc_wait(c, k, A.status);
+                const int ncols = min(S::kCols, A.GW - t * S::kCols);
+                ok = S::extra_wait(c, bt, A.status) && S::acc_wait(c, k, A.status);
                 if (!ok) break;
                 const uint32_t negc4 = c.extra(bt);
-                tcs::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
-                    const int col = t * tcs::kCols + ch * 32;        // proxy row index r = g_local * W + a
+                S::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
+                    const int col = t * S::kCols + ch * 32;        // proxy row index r = g_local * W + a
                     const int g_local = col / A.W, a0 = col % A.W;
                     if (g_local != cur_g) {                          // a head is complete: publish its mass
                         if (cur_g >= 0) {
@@ -260,7 +262,7 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                         cg += x;
                     }
                 });
-                tcs::acc_release(c);
+                S::acc_release(c);
             }
             if (ok && cur_g >= 0) {
                 const float tot = warp_sum(cg);
@@ -269,12 +271,12 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
             // the two column halves of a key meet: the upper one hands its partial sum over (kept even after a
             // wait ran out, so that the partner warp is never left waiting)
             if (c.colhalf == 1) tc::sts32(xch, imp);
-            tcs::pair_sync(c);
+            S::pair_sync(c);
             if (c.colhalf == 0 && ok && key < A.L) A.importance[(int64_t)uh * A.L + key] = (imp + tc::lds32(pxch)) / (float)A.G;   // group mean
-            tcs::pair_sync(c);
+            S::pair_sync(c);
         }
     }
-    tcs::teardown(c);
+    S::teardown(c);
 }
 
 }  // namespace flowmm
