@@ -102,14 +102,16 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
 #pragma unroll
                             for (int j = 0; j < 32; ++j) raw[j] = __uint_as_float(acc[j]);
                             mx = fmaxf(max32(raw) * A.scale_log2, m);
-                            const float neg = -mx;
+                            const float2 neg2 = make_float2(-mx, -mx), sc2 = make_float2(A.scale_log2, A.scale_log2);
+                            float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
 #pragma unroll
                             for (int j = 0; j < 32; j += 4) {
-                                add0 += tc::ex2(fmaf(raw[j], A.scale_log2, neg));
-                                add1 += tc::ex2(fmaf(raw[j + 1], A.scale_log2, neg));
-                                add2 += tc::ex2(fmaf(raw[j + 2], A.scale_log2, neg));
-                                add3 += tc::ex2_fma(fmaf(raw[j + 3], A.scale_log2, neg));     // every fourth one on the FMA pipe
+                                const float2 x01 = tc::ffma2(make_float2(raw[j], raw[j + 1]), sc2, neg2);
+                                const float2 x23 = tc::ffma2(make_float2(raw[j + 2], raw[j + 3]), sc2, neg2);
+                                a01 = tc::fadd2(a01, make_float2(tc::ex2(x01.x), tc::ex2(x01.y)));
+                                a23 = tc::fadd2(a23, make_float2(tc::ex2(x23.x), tc::ex2_fma(x23.y)));   // every fourth one on the FMA pipe
                             }
+                            add0 = a01.x; add1 = a01.y; add2 = a23.x; add3 = a23.y;
                         } else {
                             float s[32];
 #pragma unroll
@@ -234,22 +236,30 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                         cur_g = g_local;
                     }
                     float pr[32];
+                    const float2 sc2 = make_float2(A.scale_log2, A.scale_log2);
 #pragma unroll
                     for (int q4 = 0; q4 < 8; ++q4) {
                         const float4 n4 = tc::lds128(negc4 + (ch * 8 + q4) * 16);
-                        pr[4 * q4 + 0] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 0]), A.scale_log2, n4.x));
-                        pr[4 * q4 + 1] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 1]), A.scale_log2, n4.y));
-                        pr[4 * q4 + 2] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 2]), A.scale_log2, n4.z));
-                        pr[4 * q4 + 3] = tc::ex2(fmaf(__uint_as_float(acc[4 * q4 + 3]), A.scale_log2, n4.w));
+                        const float2 x01 = tc::ffma2(make_float2(__uint_as_float(acc[4 * q4 + 0]), __uint_as_float(acc[4 * q4 + 1])),
+                                                     sc2, make_float2(n4.x, n4.y));
+                        const float2 x23 = tc::ffma2(make_float2(__uint_as_float(acc[4 * q4 + 2]), __uint_as_float(acc[4 * q4 + 3])),
+                                                     sc2, make_float2(n4.z, n4.w));
+                        pr[4 * q4 + 0] = tc::ex2(x01.x);
+                        pr[4 * q4 + 1] = tc::ex2(x01.y);
+                        pr[4 * q4 + 2] = tc::ex2(x23.x);
+                        pr[4 * q4 + 3] = tc::ex2(x23.y);
                     }
                     if (masked_tile) {                               // causal mask inside the window, and keys >= L
 #pragma unroll
                         for (int j = 0; j < 32; ++j) pr[j] = (key <= first_proxy + a0 + j) ? pr[j] : 0.f;
                     }
-                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                    float2 s01 = make_float2(0.f, 0.f), s23 = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4) { s0 += pr[j]; s1 += pr[j + 1]; s2 += pr[j + 2]; s3 += pr[j + 3]; }
-                    const float csum = (s0 + s1) + (s2 + s3);
+                    for (int j = 0; j < 32; j += 4) {
+                        s01 = tc::fadd2(s01, make_float2(pr[j], pr[j + 1]));
+                        s23 = tc::fadd2(s23, make_float2(pr[j + 2], pr[j + 3]));
+                    }
+                    const float csum = (s01.x + s01.y) + (s23.x + s23.y);
                     imp += csum;
                     // proxy tokens of the other modality than this key's
                     const uint32_t wm = a0 < 32 ? wbits[0] : a0 < 64 ? wbits[1] : a0 < 96 ? wbits[2] : wbits[3];
