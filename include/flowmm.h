@@ -194,6 +194,15 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
  * (FLOWMM_OK, or the first error a kernel recorded) and clears it. */
 flowmm_status flowmm_last_device_status(void *ws, void *cuda_stream);
 
+/*
+ * Self-test of the bounded device-side waits (every mbarrier wait inside the tensor-core kernels
+ * gives up after about two seconds instead of hanging the GPU).  Enqueues one small kernel whose
+ * threads wait for an event that never comes; it returns by itself after the limit and leaves
+ * FLOWMM_ERR_TIMEOUT in the status word at the start of `ws`, which flowmm_last_device_status then
+ * reports and clears.  The CUDA context stays usable.
+ */
+flowmm_status flowmm_selftest_wait_timeout(void *ws, void *cuda_stream);
+
 /* Number of kernels the most recent compute entry point of this thread enqueued. */
 int32_t flowmm_last_launch_count(void);
 

@@ -28,7 +28,7 @@ PATH_AUTO, PATH_SIMT = 0, 1
 EXPORTS = (
     "flowmm_workspace_bytes", "flowmm_score", "flowmm_layer_flow", "flowmm_select", "flowmm_match", "flowmm_merge",
     "flowmm_compress_layer", "flowmm_last_device_status", "flowmm_last_launch_count", "flowmm_status_string",
-    "flowmm_profile_enable", "flowmm_profile_read", "flowmm_merge_static",
+    "flowmm_profile_enable", "flowmm_profile_read", "flowmm_merge_static", "flowmm_selftest_wait_timeout",
 )
 
 
@@ -119,6 +119,7 @@ def load() -> ctypes.CDLL:
         for name in EXPORTS[:8]:
             getattr(lib, name).restype = ctypes.c_int
         lib.flowmm_merge_static.restype = ctypes.c_int
+        lib.flowmm_selftest_wait_timeout.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -213,6 +214,11 @@ def flowmm_compress_layer(p: Params, q_win, k, v, modality, k_out, v_out, ws, im
 
 def flowmm_last_device_status(ws) -> int:
     return int(load().flowmm_last_device_status(_p(ws), _stream()))
+
+
+def flowmm_selftest_wait_timeout(ws):
+    """Enqueue the kernel whose wait runs out; flowmm_last_device_status(ws) then reports TIMEOUT (8)."""
+    _check(load().flowmm_selftest_wait_timeout(_p(ws), _stream()), "flowmm_selftest_wait_timeout")
 
 
 def flowmm_last_launch_count() -> int:

@@ -605,6 +605,34 @@ const char *flowmm_status_string(flowmm_status s) {
 
 }  // extern "C"
 
+// ---- bounded-wait self-test ----------------------------------------------------------------------
+namespace {
+// One CTA waits on an mbarrier phase that nothing completes, with the same bounded wait the
+// tensor-core kernels use: after the limit the first waiter records FLOWMM_ERR_TIMEOUT, raises the
+// CTA's abort flag, and every thread returns.
+__global__ void wait_timeout_selftest_kernel(int *status) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        tc::mbar_init(tc::smem_u32(&bar), 1);
+        tc::mbar_init_fence();
+    }
+    __syncthreads();
+    tc::mbar_wait(tc::smem_u32(&bar), 0, &abort_flag, status);
+}
+}  // namespace
+
+extern "C" flowmm_status flowmm_selftest_wait_timeout(void *ws, void *cuda_stream) {
+    profile_begin(static_cast<cudaStream_t>(cuda_stream));
+    if (!ws) return FLOWMM_ERR_NULL;
+    FLOWMM_TRY(check_device());
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    wait_timeout_selftest_kernel<<<1, 64, 0, st>>>(static_cast<int *>(ws));
+    FLOWMM_LAUNCHED("wait_timeout_selftest");
+    return FLOWMM_OK;
+}
+
 // ---- merge without caller scratch --------------------------------------------------------------
 // Scratch of flowmm_merge_static: lives in the library image, one copy per GPU that loads it.
 static __device__ __align__(256) unsigned char g_merge_static_scratch[FLOWMM_MERGE_STATIC_BYTES];

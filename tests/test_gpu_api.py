@@ -65,3 +65,21 @@ def test_errors_are_reported_not_computed():
     F.flowmm_score(fp, q, k, m, imp, cross, ws)
     assert F.flowmm_last_launch_count() >= 2
     torch.cuda.synchronize()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
+    """No kernel here can hang the GPU: a wait nothing satisfies gives up after its limit, the status
+    word says so, and the next call works as if nothing had happened."""
+    fp = F.Params(1, 4, 2, 128, 300, 32, 30, dtype=F.BF16)
+    ws = F.alloc_workspace(fp)
+    F.flowmm_selftest_wait_timeout(ws)
+    assert F.flowmm_last_device_status(ws) == 8            # FLOWMM_ERR_TIMEOUT
+    assert F.flowmm_last_device_status(ws) == 0            # reading it cleared it
+    rng = np.random.default_rng(5)
+    q = to_dev(inputs.round_to_bf16(rng.standard_normal((1, 4, 32, 128)).astype(np.float32)), F.BF16)
+    k = to_dev(inputs.round_to_bf16(rng.standard_normal((1, 2, 300, 128)).astype(np.float32)), F.BF16)
+    v = to_dev(inputs.round_to_bf16(rng.standard_normal((1, 2, 300, 128)).astype(np.float32)), F.BF16)
+    m = torch.from_numpy((rng.random((1, 300)) < 0.5).astype(np.uint8)).cuda()
+    out = F.compress_layer_alloc(fp, q, k, v, m, ws=ws)
+    assert F.flowmm_last_device_status(ws) == 0
+    assert torch.isfinite(out["k_out"].float()).all()
