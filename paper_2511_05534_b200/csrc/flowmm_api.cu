@@ -129,7 +129,7 @@ Layout make_layout(const flowmm_params &p) {
         y.tc_n_chunk = (key_tiles + y.tc_tiles_per_chunk - 1) / y.tc_tiles_per_chunk;
         y.gw_pad = (int)((G * W + tcs::Big::kCols - 1) / tcs::Big::kCols * tcs::Big::kCols);
     }
-    const size_t max_chunk1 = (size_t)(y.n_chunk1 > 2 * y.tc_n_chunk ? y.n_chunk1 : 2 * y.tc_n_chunk);
+    const size_t max_chunk1 = (size_t)(y.n_chunk1 > 4 * y.tc_n_chunk ? y.n_chunk1 : 4 * y.tc_n_chunk);
     const size_t max_chunk2 = (size_t)(y.n_chunk2 > 8 * y.n_rt ? y.n_chunk2 : 8 * y.n_rt);
     y.row_part = take(U * Hq * W * max_chunk1 * 8);
     y.cross_part = take(U * Hq * max_chunk2 * 4);
@@ -241,7 +241,7 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     score_stats_tc_kernel<tcs::Big><<<a.n_items1 < sms ? a.n_items1 : sms, tcs::kThreads, tcs::Big::kSmemBytes, st>>>(qa, k256, a);
     FLOWMM_LAUNCHED("score_stats_tc");
     const int n_negc = UH * a.GWpad;
-    score_combine_kernel<<<(n_negc + 255) / 256, 256, 0, st>>>(a.row_part, 2 * a.n_chunk, a.GW, a.GWpad, UH, a.negc);
+    score_combine_kernel<<<(n_negc + 255) / 256, 256, 0, st>>>(a.row_part, 4 * a.n_chunk, a.GW, a.GWpad, UH, a.negc);
     FLOWMM_LAUNCHED("score_combine");
     if (small2)
         score_colsum_tc_kernel<tcs::Small><<<a.n_items2 < sms ? a.n_items2 : sms, tcs::kThreads, tcs::Small::kSmemBytes, st>>>(k128, qb, a);

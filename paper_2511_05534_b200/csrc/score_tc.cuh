@@ -19,7 +19,7 @@
 namespace flowmm {
 
 struct ScoreTcArgs {
-    float2 *row_part;            // [UH*GW, 2*n_chunk] (max, sum) per proxy row, key chunk and column half, log2 domain
+    float2 *row_part;            // [UH*GW, 4*n_chunk] (max, sum) per proxy row, key chunk and column quarter, log2 domain
     float *negc;                 // [UH, GWpad] -(row max + log2 row sum); very negative for padding rows
     const uint8_t *modality;     // [U, L]
     float *importance;           // [UH, L]
@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(tcs::kThreads, 1)
 score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                       const ScoreTcArgs A) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const typename S::Ctx c = S::setup(smem_raw, &q_map, &k_map, A.status);
+    const typename S::Ctx c = S::setup(smem_raw, &q_map, &k_map, A.status, 0, 16);
     if (!c.ok) return;
     auto plan = [&](int item) {
         tcs::TilePlan p;
@@ -75,67 +75,76 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
     } else if (c.warp == 1) {
         if (c.lane == 0) S::mma_issuer(c, A.n_items1, plan, A.status);
     } else {
-        const int row_in_half = c.quarter * 32 + c.lane;
-        int k = 0;
+        // all sixteen warps drain one accumulator at a time: a warp owns 32 lanes x a quarter of the columns of
+        // BOTH halves, so the tensor core refills one half while the other is being read
+        const int row_in_half = c.quarter * 32 + c.lane, colq = (c.warp - 2) >> 2;
+        int kh[2] = {0, 0};
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items1; item += gridDim.x) {
             const tcs::TilePlan p = plan(item);
-            if (p.empty() || c.group >= p.n_halves) continue;
+            if (p.empty()) continue;
             const int kc = item % A.n_chunk, qt = (item / A.n_chunk) % A.n_qt, uh = item / (A.n_chunk * A.n_qt);
-            const int r = qt * tcs::kItemRows + c.group * tcs::kRows + row_in_half;
-            const bool valid_row = r < A.GW;
-            const bool warp_has_rows = qt * tcs::kItemRows + c.group * tcs::kRows + c.quarter * 32 < A.GW;
-            const int pa = A.L - A.W + (r % A.W);                    // last key this proxy row may see
-            float m = kNegBig, l = 0.f;
-            for (int t = 0; ok && t < p.n_tiles; ++t, ++k) {
-                ok = S::acc_wait(c, k, A.status);
-                if (!ok) break;
+            float m[2] = {kNegBig, kNegBig}, l[2] = {0.f, 0.f};
+            for (int t = 0; ok && t < p.n_tiles; ++t) {
                 const int kb = p.b1 + t * S::kCols;
                 const int ncols = min(S::kCols, p.cols_total - t * S::kCols);
-                if (warp_has_rows) {
-                    S::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
-                        const int k0 = kb + ch * 32;
-                        float mx;
-                        float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
-                        if (k0 + 32 <= A.L - A.W + 1) {              // no key of this chunk is masked for any row
-                            float raw[32];
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) raw[j] = __uint_as_float(acc[j]);
-                            mx = fmaxf(max32(raw) * A.scale_log2, m);
-                            const float2 neg2 = make_float2(-mx, -mx), sc2 = make_float2(A.scale_log2, A.scale_log2);
-                            float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
+                for (int h = 0; h < 2; ++h) {
+                    if (h >= p.n_halves || !ok) continue;
+                    ok = S::acc_wait_h(c, h, kh[h]++, A.status);
+                    if (!ok) continue;
+                    const int r0 = qt * tcs::kItemRows + h * tcs::kRows;
+                    const int pa = A.L - A.W + ((r0 + row_in_half) % A.W);   // last key this proxy row may see
+                    if (r0 + c.quarter * 32 < A.GW) {
+                        S::for_each_chunk_q(c, h, colq, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
+                            const int k0 = kb + ch * 32;
+                            float mx;
+                            float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
+                            if (k0 + 32 <= A.L - A.W + 1) {              // no key of this chunk is masked for any row
+                                float raw[32];
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                const float2 x01 = tc::ffma2(make_float2(raw[j], raw[j + 1]), sc2, neg2);
-                                const float2 x23 = tc::ffma2(make_float2(raw[j + 2], raw[j + 3]), sc2, neg2);
-                                a01 = tc::fadd2(a01, make_float2(tc::ex2(x01.x), tc::ex2(x01.y)));
-                                a23 = tc::fadd2(a23, make_float2(tc::ex2(x23.x), tc::ex2_fma(x23.y)));   // every fourth one on the FMA pipe
+                                for (int j = 0; j < 32; ++j) raw[j] = __uint_as_float(acc[j]);
+                                mx = fmaxf(max32(raw) * A.scale_log2, m[h]);
+                                const float2 neg2 = make_float2(-mx, -mx), sc2 = make_float2(A.scale_log2, A.scale_log2);
+                                float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4) {
+                                    const float2 x01 = tc::ffma2(make_float2(raw[j], raw[j + 1]), sc2, neg2);
+                                    const float2 x23 = tc::ffma2(make_float2(raw[j + 2], raw[j + 3]), sc2, neg2);
+                                    a01 = tc::fadd2(a01, make_float2(tc::ex2(x01.x), tc::ex2(x01.y)));
+                                    a23 = tc::fadd2(a23, make_float2(tc::ex2(x23.x), tc::ex2_fma(x23.y)));   // every fourth one on the FMA pipe
+                                }
+                                add0 = a01.x; add1 = a01.y; add2 = a23.x; add3 = a23.y;
+                            } else {
+                                float s[32];
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    s[j] = (k0 + j <= pa) ? __uint_as_float(acc[j]) * A.scale_log2 : kNegBig;
+                                mx = fmaxf(max32(s), m[h]);
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4) {        // masked entries sit ~1e30 below: exp2 gives 0
+                                    add0 += tc::ex2(s[j] - mx);
+                                    add1 += tc::ex2(s[j + 1] - mx);
+                                    add2 += tc::ex2(s[j + 2] - mx);
+                                    add3 += tc::ex2(s[j + 3] - mx);
+                                }
                             }
-                            add0 = a01.x; add1 = a01.y; add2 = a23.x; add3 = a23.y;
-                        } else {
-                            float s[32];
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                s[j] = (k0 + j <= pa) ? __uint_as_float(acc[j]) * A.scale_log2 : kNegBig;
-                            mx = fmaxf(max32(s), m);
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) {        // masked entries sit ~1e30 below: exp2 gives 0
-                                add0 += tc::ex2(s[j] - mx);
-                                add1 += tc::ex2(s[j + 1] - mx);
-                                add2 += tc::ex2(s[j + 2] - mx);
-                                add3 += tc::ex2(s[j + 3] - mx);
-                            }
-                        }
-                        float add = (add0 + add1) + (add2 + add3);
-                        if (mx < 0.5f * kNegBig) add = 0.f;          // nothing visible yet: exp2(0) terms are not real
-                        l = l * tc::ex2(m - mx) + add;
-                        m = mx;
-                    });
+                            float add = (add0 + add1) + (add2 + add3);
+                            if (mx < 0.5f * kNegBig) add = 0.f;          // nothing visible yet: exp2(0) terms are not real
+                            l[h] = l[h] * tc::ex2(m[h] - mx) + add;
+                            m[h] = mx;
+                        });
+                    }
+                    S::acc_release_h(c, h);
                 }
-                S::acc_release(c);
             }
             if (!ok) break;
-            if (valid_row) A.row_part[((int64_t)uh * A.GW + r) * (2 * A.n_chunk) + 2 * kc + c.colhalf] = make_float2(m, l);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int r = qt * tcs::kItemRows + h * tcs::kRows + row_in_half;
+                if (h < p.n_halves && r < A.GW)
+                    A.row_part[((int64_t)uh * A.GW + r) * (4 * A.n_chunk) + 4 * kc + colq] = make_float2(m[h], l[h]);
+            }
         }
     }
     S::teardown(c);

@@ -89,7 +89,7 @@ struct Skel {
 
     // `a_readers`: epilogue warps per half that read the A stage themselves and release it with a_release().
     static __device__ __forceinline__ Ctx setup(uint8_t *smem_raw, const CUtensorMap *ma, const CUtensorMap *mb,
-                                                int *status, int a_readers = 0) {
+                                                int *status, int a_readers = 0, int acc_arrivals = 8) {
         Ctx c;
         c.base = tc::smem_u32(smem_raw);
         c.bars = c.base + kSmemBar;
@@ -110,7 +110,7 @@ struct Skel {
             for (int i = 0; i < kNumBars; ++i) {
                 int count = 1;
                 if (i >= kBarAEmpty && i < kBarBFull) count = 1 + a_readers;
-                if (i >= kBarAccEmpty && i < kBarXFull) count = 8;       // one arrival per epilogue warp of the half
+                if (i >= kBarAccEmpty && i < kBarXFull) count = acc_arrivals;   // one arrival per epilogue warp that reads the half
                 tc::mbar_init(c.bar(i), count);
             }
             *c.abort_flag = 0;
@@ -274,6 +274,29 @@ struct Skel {
             tc::tmem_ld16(c.tmem_base + c.group * NB + b * 16 + ((uint32_t)(c.quarter * 32) << 16), a);
             tc::tmem_ld_wait(a);
             f(b, a);
+        }
+    }
+    // The same for epilogues in which all sixteen warps drain one accumulator at a time (warp = 32 lanes x
+    // a quarter of the columns, both halves in turn): explicit half index, `k` = tiles of that half so far.
+    static __device__ __forceinline__ bool acc_wait_h(const Ctx &c, int h, int k, int *status) {
+        const bool ok = tc::mbar_wait(c.bar(kBarAccFull + h), k & 1, c.abort_flag, status);
+        tc::tc_fence_after();
+        return ok;
+    }
+    static __device__ __forceinline__ void acc_release_h(const Ctx &c, int h) {
+        tc::tc_fence_before();
+        __syncwarp();
+        if (c.lane == 0) tc::mbar_arrive(c.bar(kBarAccEmpty + h));
+    }
+    template <class F>
+    static __device__ __forceinline__ void for_each_chunk_q(const Ctx &c, int h, int colq, int n_chunks, F &&f) {
+        constexpr int kPer = NB / 128;
+        const int hi = min(n_chunks, kPer * colq + kPer);
+        for (int ch = kPer * colq; ch < hi; ++ch) {
+            uint32_t a[32];
+            tc::tmem_ld32(c.tmem_base + h * NB + ch * 32 + ((uint32_t)(c.quarter * 32) << 16), a);
+            tc::tmem_ld_wait(a);
+            f(ch, a);
         }
     }
     // Meeting point of the two warps that share rows (same half, same lanes, other columns).
