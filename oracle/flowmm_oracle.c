@@ -26,6 +26,8 @@
  *               pivots and its argmax                                   (Eq. 9, Eq. 10)
  *   merge       weighted consolidation of non-pivots into their pivots and
  *               compaction to B rows                                    (Eq. 5)
+ *   decode      (the step after the path) one new query's attention over the
+ *               cache, full or compressed                               (Eq. 4)
  *
  * Readings where the paper is silent (all listed in the design notes): group
  * mean for GQA importance; rho restricted to the proxy rows; rho == theta is
@@ -303,6 +305,47 @@ int flowmm_oracle_merge(const oracle_params *p, const float *k, const float *v,
                 if (weight_sum) weight_sum[uh * (size_t)B + s] = z[s];
             }
             free(z);
+        }
+    }
+    return 0;
+}
+
+/*
+ * Decode-step attention over a (compressed or full) cache, Eq. 4: for the one new query of head g,
+ * o = softmax(q . K^T / sqrt(d)) V over the n_keys rows of its KV head h = g / G.  No mask: the
+ * query comes after every cached token.  scale 0 selects 1/sqrt(head_dim).
+ *   q   [U, Hq, D]      k, v [U, Hkv, n_keys, D]      out [U, Hq, D] (double)
+ */
+int flowmm_oracle_decode_attention(int32_t n_units, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                   int32_t n_keys, double scale, const float *q, const float *k, const float *v,
+                                   double *out)
+{
+    if (n_units < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads != 0 || head_dim < 1 || n_keys < 1)
+        return 1;
+    const int G = n_q_heads / n_kv_heads, D = head_dim, N = n_keys;
+    if (scale == 0.0) scale = 1.0 / sqrt((double)D);
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int u = 0; u < n_units; ++u) {
+        for (int g = 0; g < n_q_heads; ++g) {
+            const int h = g / G;
+            const float *qg = q + ((size_t)u * n_q_heads + g) * D;
+            const float *kh = k + ((size_t)u * n_kv_heads + h) * (size_t)N * D;
+            const float *vh = v + ((size_t)u * n_kv_heads + h) * (size_t)N * D;
+            double *o = out + ((size_t)u * n_q_heads + g) * D;
+            double *s = (double *)malloc(sizeof(double) * (size_t)N);
+            double mx = -INFINITY;
+            for (int i = 0; i < N; ++i) {
+                s[i] = scale * dotd(qg, kh + (size_t)i * D, D);
+                if (s[i] > mx) mx = s[i];
+            }
+            double z = 0.0;
+            for (int i = 0; i < N; ++i) { s[i] = exp(s[i] - mx); z += s[i]; }
+            for (int c = 0; c < D; ++c) o[c] = 0.0;
+            for (int i = 0; i < N; ++i) {
+                const double a = s[i] / z;
+                for (int c = 0; c < D; ++c) o[c] += a * (double)vh[(size_t)i * D + c];
+            }
+            free(s);
         }
     }
     return 0;

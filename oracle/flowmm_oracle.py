@@ -203,3 +203,18 @@ def compress_layer(p: OracleParams, q, k, v, modality, forced: Optional[Dict[str
         ko, vo, z = merge(p, k, v, out["retained"], out["evicted"], out["match"], out["match_sim"])
         out["k_out"], out["v_out"], out["weight_sum"] = ko, vo, z
     return out
+
+
+def decode_attention(q, k, v, scale: float = 0.0) -> np.ndarray:
+    """Eq. 4 for one decode step over a cache: q [U,Hq,D], k, v [U,Hkv,N,D] -> out [U,Hq,D] float64."""
+    q, k, v = _f32(q), _f32(k), _f32(v)
+    U, Hq, D = q.shape
+    Hkv, N = k.shape[1], k.shape[2]
+    assert k.shape == (U, Hkv, N, D) and v.shape == k.shape
+    out = np.zeros((U, Hq, D), dtype=np.float64)
+    rc = _load().flowmm_oracle_decode_attention(ctypes.c_int32(U), ctypes.c_int32(Hq), ctypes.c_int32(Hkv),
+                                                ctypes.c_int32(D), ctypes.c_int32(N), ctypes.c_double(scale),
+                                                _ptr(q), _ptr(k), _ptr(v), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle decode_attention: bad shape (code %d)" % rc)
+    return out
