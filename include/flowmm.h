@@ -190,6 +190,29 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
                                     int32_t *match, float *match_sim,
                                     void *ws, size_t ws_bytes, void *cuda_stream);
 
+/*
+ * The step after the compression path: decode-time attention of one new query per query head over a
+ * cache of n_keys rows, Eq. 4 - o = softmax(q . K^T * scale) V - for the full cache or for the
+ * compressed one that flowmm_compress_layer wrote.  Every cache row is read once for all G query
+ * heads of its KV head.
+ *   q   [U, Hq, D]  dense, element type `dtype`
+ *   k,v [U, Hkv, n_keys, D] with the element strides given (unit, head, token); head_dim contiguous
+ *   out [U, Hq, D]  f32
+ * n_q_heads / n_kv_heads must be at most 8; head_dim 64 or 128.  Scratch: flowmm_decode_workspace_bytes.
+ * Same conventions as above (device pointers, caller-owned memory, asynchronous on the stream).
+ */
+typedef struct {
+    int32_t n_units, n_q_heads, n_kv_heads, head_dim;
+    int32_t n_keys;                     /* rows of the cache to attend to (L, or B after compression) */
+    int32_t dtype;                      /* flowmm_dtype of q, k, v */
+    float softmax_scale;                /* 0 selects 1/sqrt(head_dim) */
+    int64_t k_stride[3], v_stride[3];   /* element strides of (unit, head, token) */
+} flowmm_decode_params;
+
+flowmm_status flowmm_decode_workspace_bytes(const flowmm_decode_params *p, size_t *bytes);
+flowmm_status flowmm_decode_attention(const flowmm_decode_params *p, const void *q, const void *k, const void *v,
+                                      float *out, void *ws, size_t ws_bytes, void *cuda_stream);
+
 /* Waits for `cuda_stream`, then returns the device status word at the start of `ws`
  * (FLOWMM_OK, or the first error a kernel recorded) and clears it. */
 flowmm_status flowmm_last_device_status(void *ws, void *cuda_stream);

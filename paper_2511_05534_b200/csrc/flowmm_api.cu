@@ -9,6 +9,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "decode.cuh"
 #include "match_tc.cuh"
 #include "score_tc.cuh"
 #include "select_merge.cuh"
@@ -604,6 +605,87 @@ const char *flowmm_status_string(flowmm_status s) {
 }
 
 }  // extern "C"
+
+// ---- decode-step attention over a cache ---------------------------------------------------------
+namespace {
+
+flowmm_status validate_decode(const flowmm_decode_params *p) {
+    if (!p) return FLOWMM_ERR_NULL;
+    if (p->n_units < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_keys < 1) return FLOWMM_ERR_SHAPE;
+    if (p->n_q_heads % p->n_kv_heads != 0 || p->n_q_heads / p->n_kv_heads > 8) return FLOWMM_ERR_SHAPE;
+    if (p->head_dim != 64 && p->head_dim != 128) return FLOWMM_ERR_SHAPE;
+    if ((int64_t)p->n_units * p->n_kv_heads > 65535) return FLOWMM_ERR_SHAPE;
+    if (p->dtype != FLOWMM_F32 && p->dtype != FLOWMM_BF16) return FLOWMM_ERR_DTYPE;
+    if (!(p->softmax_scale >= 0.f)) return FLOWMM_ERR_SHAPE;
+    return FLOWMM_OK;
+}
+
+// key ranges per (unit, KV head): enough CTAs for about four per SM, at least 64 keys each
+void decode_split(const flowmm_decode_params &p, int &n_split, int &keys_per_split) {
+    const int uh = p.n_units * p.n_kv_heads;
+    int want = (4 * 148 + uh - 1) / uh;
+    const int max_split = (p.n_keys + 63) / 64;
+    want = want < 1 ? 1 : (want > max_split ? max_split : want);
+    keys_per_split = (p.n_keys + want - 1) / want;
+    n_split = (p.n_keys + keys_per_split - 1) / keys_per_split;
+}
+
+template <typename T, int D>
+flowmm_status launch_decode(const DecodeArgs &a, int uh, int n_q, cudaStream_t st) {
+    constexpr int groups = kDecThreads / (D / Elem<T>::kVec);
+    const dim3 grid(a.n_split, uh);
+    const int gp = a.G <= 1 ? 1 : a.G <= 2 ? 2 : a.G <= 4 ? 4 : 8;
+    const size_t smem = (size_t)groups * gp * (D + 2) * sizeof(float);
+    switch (gp) {
+        case 1: decode_partial_kernel<T, D, 1><<<grid, kDecThreads, smem, st>>>(a); break;
+        case 2: decode_partial_kernel<T, D, 2><<<grid, kDecThreads, smem, st>>>(a); break;
+        case 4: decode_partial_kernel<T, D, 4><<<grid, kDecThreads, smem, st>>>(a); break;
+        default: decode_partial_kernel<T, D, 8><<<grid, kDecThreads, smem, st>>>(a); break;
+    }
+    FLOWMM_LAUNCHED("decode_partial");
+    decode_combine_kernel<D><<<n_q, D, 0, st>>>(a);
+    FLOWMM_LAUNCHED("decode_combine");
+    return FLOWMM_OK;
+}
+
+}  // namespace
+
+extern "C" flowmm_status flowmm_decode_workspace_bytes(const flowmm_decode_params *p, size_t *bytes) {
+    if (!bytes) return FLOWMM_ERR_NULL;
+    FLOWMM_TRY(validate_decode(p));
+    int n_split, kps;
+    decode_split(*p, n_split, kps);
+    *bytes = align256((size_t)p->n_units * p->n_kv_heads * n_split * (p->n_q_heads / p->n_kv_heads) *
+                      (p->head_dim + 2) * sizeof(float));
+    return FLOWMM_OK;
+}
+
+extern "C" flowmm_status flowmm_decode_attention(const flowmm_decode_params *p, const void *q, const void *k,
+                                                 const void *v, float *out, void *ws, size_t ws_bytes,
+                                                 void *cuda_stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    profile_begin(st);
+    FLOWMM_TRY(validate_decode(p));
+    if (!q || !k || !v || !out || !ws) return FLOWMM_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !strides_ok(p->k_stride, p->head_dim) ||
+        !strides_ok(p->v_stride, p->head_dim) || (reinterpret_cast<uintptr_t>(ws) & 255))
+        return FLOWMM_ERR_ALIGN;
+    size_t need = 0;
+    FLOWMM_TRY(flowmm_decode_workspace_bytes(p, &need));
+    if (ws_bytes < need) return FLOWMM_ERR_WORKSPACE;
+    FLOWMM_TRY(check_device());
+    DecodeArgs a;
+    a.q = q; a.k = k; a.v = v; a.part = static_cast<float *>(ws); a.out = out;
+    a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads; a.G = p->n_q_heads / p->n_kv_heads; a.N = p->n_keys;
+    decode_split(*p, a.n_split, a.keys_per_split);
+    const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.f / sqrtf((float)p->head_dim);
+    a.scale_log2 = scale * kLog2e;
+    for (int i = 0; i < 3; ++i) { a.ks[i] = p->k_stride[i]; a.vs[i] = p->v_stride[i]; }
+    const int uh = p->n_units * p->n_kv_heads, n_q = p->n_units * p->n_q_heads;
+    if (p->dtype == FLOWMM_BF16)
+        return p->head_dim == 128 ? launch_decode<__nv_bfloat16, 128>(a, uh, n_q, st) : launch_decode<__nv_bfloat16, 64>(a, uh, n_q, st);
+    return p->head_dim == 128 ? launch_decode<float, 128>(a, uh, n_q, st) : launch_decode<float, 64>(a, uh, n_q, st);
+}
 
 // ---- bounded-wait self-test ----------------------------------------------------------------------
 namespace {
