@@ -198,7 +198,10 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
  *   q   [U, Hq, D]  dense, element type `dtype`
  *   k,v [U, Hkv, n_keys, D] with the element strides given (unit, head, token); head_dim contiguous
  *   out [U, Hq, D]  f32
- * n_q_heads / n_kv_heads must be at most 8; head_dim 64 or 128.  Scratch: flowmm_decode_workspace_bytes.
+ * n_q_heads / n_kv_heads must be at most 8; head_dim 64 or 128.  Scratch: flowmm_decode_workspace_bytes
+ * (its first word is a device status like the compression workspace's, see flowmm_last_device_status).
+ * `path` as in flowmm_params: AUTO runs both contractions on the tensor cores (tcgen05) when dtype is
+ * bf16 and head_dim is 128, and SIMT fp32 kernels otherwise; SIMT forces the latter.
  * Same conventions as above (device pointers, caller-owned memory, asynchronous on the stream).
  */
 typedef struct {
@@ -206,6 +209,7 @@ typedef struct {
     int32_t n_keys;                     /* rows of the cache to attend to (L, or B after compression) */
     int32_t dtype;                      /* flowmm_dtype of q, k, v */
     float softmax_scale;                /* 0 selects 1/sqrt(head_dim) */
+    int32_t path;                       /* flowmm_path */
     int64_t k_stride[3], v_stride[3];   /* element strides of (unit, head, token) */
 } flowmm_decode_params;
 

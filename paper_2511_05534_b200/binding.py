@@ -223,33 +223,33 @@ class _CDecodeParams(ctypes.Structure):
     _fields_ = [
         ("n_units", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32), ("n_keys", ctypes.c_int32), ("dtype", ctypes.c_int32),
-        ("softmax_scale", ctypes.c_float),
+        ("softmax_scale", ctypes.c_float), ("path", ctypes.c_int32),
         ("k_stride", ctypes.c_int64 * 3), ("v_stride", ctypes.c_int64 * 3),
     ]
 
 
-def _decode_params(q, k, v, softmax_scale: float) -> _CDecodeParams:
+def _decode_params(q, k, v, softmax_scale: float, path: int) -> _CDecodeParams:
     if q.dim() != 3 or not q.is_contiguous():
         raise ValueError("q must be a contiguous [units, q_heads, head_dim] tensor")
     if k.dim() != 4 or v.dim() != 4 or k.stride(3) != 1 or v.stride(3) != 1 or k.shape != v.shape:
         raise ValueError("k, v must be [units, kv_heads, keys, head_dim] tensors with contiguous head_dim")
     dtype = BF16 if q.dtype == torch.bfloat16 else F32
-    cp = _CDecodeParams(q.shape[0], q.shape[1], k.shape[1], q.shape[2], k.shape[2], dtype, softmax_scale)
+    cp = _CDecodeParams(q.shape[0], q.shape[1], k.shape[1], q.shape[2], k.shape[2], dtype, softmax_scale, path)
     cp.k_stride = (ctypes.c_int64 * 3)(k.stride(0), k.stride(1), k.stride(2))
     cp.v_stride = (ctypes.c_int64 * 3)(v.stride(0), v.stride(1), v.stride(2))
     return cp
 
 
-def flowmm_decode_workspace_bytes(q, k, v, softmax_scale: float = 0.0) -> int:
+def flowmm_decode_workspace_bytes(q, k, v, softmax_scale: float = 0.0, path: int = PATH_AUTO) -> int:
     n = ctypes.c_size_t(0)
-    cp = _decode_params(q, k, v, softmax_scale)
+    cp = _decode_params(q, k, v, softmax_scale, path)
     _check(load().flowmm_decode_workspace_bytes(ctypes.byref(cp), ctypes.byref(n)), "flowmm_decode_workspace_bytes")
     return int(n.value)
 
 
-def flowmm_decode_attention(q, k, v, out, ws, softmax_scale: float = 0.0):
+def flowmm_decode_attention(q, k, v, out, ws, softmax_scale: float = 0.0, path: int = PATH_AUTO):
     """Eq. 4 for one new query per head over the cache rows of k, v; out [units, q_heads, head_dim] float32."""
-    cp = _decode_params(q, k, v, softmax_scale)
+    cp = _decode_params(q, k, v, softmax_scale, path)
     _check(load().flowmm_decode_attention(ctypes.byref(cp), _p(q), _p(k), _p(v), _p(out), _p(ws),
                                           ctypes.c_size_t(ws.numel()), _stream()), "flowmm_decode_attention")
 

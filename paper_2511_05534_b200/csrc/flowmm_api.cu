@@ -10,6 +10,7 @@
 
 #include "common.cuh"
 #include "decode.cuh"
+#include "decode_tc.cuh"
 #include "match_tc.cuh"
 #include "score_tc.cuh"
 #include "select_merge.cuh"
@@ -617,17 +618,38 @@ flowmm_status validate_decode(const flowmm_decode_params *p) {
     if ((int64_t)p->n_units * p->n_kv_heads > 65535) return FLOWMM_ERR_SHAPE;
     if (p->dtype != FLOWMM_F32 && p->dtype != FLOWMM_BF16) return FLOWMM_ERR_DTYPE;
     if (!(p->softmax_scale >= 0.f)) return FLOWMM_ERR_SHAPE;
+    if (p->path != FLOWMM_PATH_AUTO && p->path != FLOWMM_PATH_SIMT) return FLOWMM_ERR_SHAPE;
     return FLOWMM_OK;
 }
 
-// key ranges per (unit, KV head): enough CTAs for about four per SM, at least 64 keys each
-void decode_split(const flowmm_decode_params &p, int &n_split, int &keys_per_split) {
-    const int uh = p.n_units * p.n_kv_heads;
-    int want = (4 * 148 + uh - 1) / uh;
-    const int max_split = (p.n_keys + 63) / 64;
-    want = want < 1 ? 1 : (want > max_split ? max_split : want);
-    keys_per_split = (p.n_keys + want - 1) / want;
-    n_split = (p.n_keys + keys_per_split - 1) / keys_per_split;
+// How a call is cut into key ranges, and where its scratch lives: [status word, 256 bytes][partial records].
+struct DecodePlan {
+    bool tc;                 // tensor-core kernel (bf16, head_dim 128) or the SIMT one
+    int n_split, per_split;  // ranges per (unit, KV head); keys (SIMT) or 128-key tiles (tensor core) per range
+    size_t bytes;
+};
+
+DecodePlan decode_plan(const flowmm_decode_params &p) {
+    DecodePlan d;
+    const int uh = p.n_units * p.n_kv_heads, g = p.n_q_heads / p.n_kv_heads;
+    d.tc = p.dtype == FLOWMM_BF16 && p.head_dim == 128 && p.path != FLOWMM_PATH_SIMT;
+    if (d.tc) {
+        // two CTAs per SM; about two rounds of them when the cache is long enough, never more tiles than TMEM holds
+        const int tiles = (p.n_keys + dtc::kTile - 1) / dtc::kTile;
+        int per = (int)(((int64_t)tiles * uh + 4 * tc::sm_count() - 1) / (4 * tc::sm_count()));
+        per = per < 1 ? 1 : (per > dtc::kMaxTiles ? dtc::kMaxTiles : per);
+        d.per_split = per;
+        d.n_split = (tiles + per - 1) / per;
+    } else {
+        // enough CTAs for about four per SM, at least 64 keys each
+        int want = (4 * 148 + uh - 1) / uh;
+        const int max_split = (p.n_keys + 63) / 64;
+        want = want < 1 ? 1 : (want > max_split ? max_split : want);
+        d.per_split = (p.n_keys + want - 1) / want;
+        d.n_split = (p.n_keys + d.per_split - 1) / d.per_split;
+    }
+    d.bytes = 256 + align256((size_t)uh * d.n_split * g * (p.head_dim + 2) * sizeof(float));
+    return d;
 }
 
 template <typename T, int D>
@@ -648,15 +670,41 @@ flowmm_status launch_decode(const DecodeArgs &a, int uh, int n_q, cudaStream_t s
     return FLOWMM_OK;
 }
 
+flowmm_status launch_decode_tc(const flowmm_decode_params &p, const DecodeArgs &a, int *status, int uh, int n_q,
+                               cudaStream_t st) {
+    CUtensorMap kmap, vmap;
+    const uint64_t dims[4] = {128, (uint64_t)p.n_keys, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
+    const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
+    const uint64_t vs[3] = {(uint64_t)p.v_stride[2] * 2, (uint64_t)p.v_stride[1] * 2, (uint64_t)p.v_stride[0] * 2};
+    const uint32_t box[4] = {64, dtc::kTile, 1, 1};
+    if (!tc::make_bf16_map(&kmap, a.k, 4, dims, ks, box) || !tc::make_bf16_map(&vmap, a.v, 4, dims, vs, box))
+        return FLOWMM_ERR_CUDA;
+    static bool configured = false;      // per process; the attribute is the same on every device
+    if (!configured) {
+        if (cudaFuncSetAttribute(dtc::decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)dtc::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(dtc::decode_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+            return FLOWMM_ERR_CUDA;
+        configured = true;
+    }
+    dtc::Args t;
+    t.q = static_cast<const __nv_bfloat16 *>(a.q); t.part = a.part; t.status = status;
+    t.Hq = a.Hq; t.Hkv = a.Hkv; t.G = a.G; t.N = a.N; t.n_split = a.n_split; t.tiles_per_split = a.keys_per_split;
+    t.scale_log2 = a.scale_log2;
+    dtc::decode_tc_kernel<<<dim3(a.n_split, uh), dtc::kThreads, dtc::kSmemBytes, st>>>(kmap, vmap, t);
+    FLOWMM_LAUNCHED("decode_tc");
+    decode_combine_kernel<128><<<n_q, 128, 0, st>>>(a);
+    FLOWMM_LAUNCHED("decode_combine");
+    return FLOWMM_OK;
+}
+
 }  // namespace
 
 extern "C" flowmm_status flowmm_decode_workspace_bytes(const flowmm_decode_params *p, size_t *bytes) {
     if (!bytes) return FLOWMM_ERR_NULL;
     FLOWMM_TRY(validate_decode(p));
-    int n_split, kps;
-    decode_split(*p, n_split, kps);
-    *bytes = align256((size_t)p->n_units * p->n_kv_heads * n_split * (p->n_q_heads / p->n_kv_heads) *
-                      (p->head_dim + 2) * sizeof(float));
+    *bytes = decode_plan(*p).bytes;
     return FLOWMM_OK;
 }
 
@@ -670,18 +718,19 @@ extern "C" flowmm_status flowmm_decode_attention(const flowmm_decode_params *p, 
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !strides_ok(p->k_stride, p->head_dim) ||
         !strides_ok(p->v_stride, p->head_dim) || (reinterpret_cast<uintptr_t>(ws) & 255))
         return FLOWMM_ERR_ALIGN;
-    size_t need = 0;
-    FLOWMM_TRY(flowmm_decode_workspace_bytes(p, &need));
-    if (ws_bytes < need) return FLOWMM_ERR_WORKSPACE;
+    const DecodePlan plan = decode_plan(*p);
+    if (ws_bytes < plan.bytes) return FLOWMM_ERR_WORKSPACE;
     FLOWMM_TRY(check_device());
+    if (cudaMemsetAsync(ws, 0, 4, st) != cudaSuccess) return FLOWMM_ERR_CUDA;
     DecodeArgs a;
-    a.q = q; a.k = k; a.v = v; a.part = static_cast<float *>(ws); a.out = out;
+    a.q = q; a.k = k; a.v = v; a.part = reinterpret_cast<float *>(static_cast<char *>(ws) + 256); a.out = out;
     a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads; a.G = p->n_q_heads / p->n_kv_heads; a.N = p->n_keys;
-    decode_split(*p, a.n_split, a.keys_per_split);
+    a.n_split = plan.n_split; a.keys_per_split = plan.per_split;
     const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.f / sqrtf((float)p->head_dim);
     a.scale_log2 = scale * kLog2e;
     for (int i = 0; i < 3; ++i) { a.ks[i] = p->k_stride[i]; a.vs[i] = p->v_stride[i]; }
     const int uh = p->n_units * p->n_kv_heads, n_q = p->n_units * p->n_q_heads;
+    if (plan.tc) return launch_decode_tc(*p, a, static_cast<int *>(ws), uh, n_q, st);
     if (p->dtype == FLOWMM_BF16)
         return p->head_dim == 128 ? launch_decode<__nv_bfloat16, 128>(a, uh, n_q, st) : launch_decode<__nv_bfloat16, 64>(a, uh, n_q, st);
     return p->head_dim == 128 ? launch_decode<float, 128>(a, uh, n_q, st) : launch_decode<float, 64>(a, uh, n_q, st);

@@ -14,12 +14,12 @@ pytestmark = pytest.mark.gpu
 RTOL, ATOL = 2e-3, 2e-3      # fp32 accumulation of bf16 inputs, ex2.approx weights; values are O(1)
 
 
-def _run(q, k, v, dtype, scale=0.0):
+def _run(q, k, v, dtype, scale=0.0, path=F.PATH_AUTO):
     qd, kd, vd = to_dev(q, dtype), to_dev(k, dtype), to_dev(v, dtype)
-    out = torch.empty(q.shape, dtype=torch.float32, device="cuda")
-    ws = torch.empty(F.flowmm_decode_workspace_bytes(qd, kd, vd, scale), dtype=torch.uint8, device="cuda")
-    F.flowmm_decode_attention(qd, kd, vd, out, ws, scale)
-    torch.cuda.synchronize()
+    out = torch.full(q.shape, float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(F.flowmm_decode_workspace_bytes(qd, kd, vd, scale, path), dtype=torch.uint8, device="cuda")
+    F.flowmm_decode_attention(qd, kd, vd, out, ws, scale, path)
+    assert F.flowmm_last_device_status(ws) == 0
     return out.cpu().numpy().astype(np.float64)
 
 
@@ -33,9 +33,10 @@ def test_ragged_shapes_against_oracle(dtype, D):
         v = rng.standard_normal((U, Hkv, N, D)).astype(np.float32)
         if dtype == F.BF16:
             q, k, v = inputs.round_to_bf16(q), inputs.round_to_bf16(k), inputs.round_to_bf16(v)
-        got = _run(q, k, v, dtype)
         ref = O.decode_attention(q, k, v)
-        assert np.allclose(got, ref, rtol=RTOL, atol=ATOL), (U, Hq, Hkv, N, np.abs(got - ref).max())
+        for path in (F.PATH_AUTO, F.PATH_SIMT):          # AUTO is the tensor-core kernel for bf16 at head_dim 128
+            got = _run(q, k, v, dtype, path=path)
+            assert np.allclose(got, ref, rtol=RTOL, atol=ATOL), (U, Hq, Hkv, N, path, np.abs(got - ref).max())
 
 
 def test_peaked_attention_and_explicit_scale():
@@ -44,7 +45,8 @@ def test_peaked_attention_and_explicit_scale():
     k = inputs.round_to_bf16(rng.standard_normal((1, 2, 700, 128)).astype(np.float32))
     v = inputs.round_to_bf16(rng.standard_normal((1, 2, 700, 128)).astype(np.float32))
     for scale in (0.0, 0.5):
-        assert np.allclose(_run(q, k, v, F.BF16, scale), O.decode_attention(q, k, v, scale), rtol=RTOL, atol=ATOL)
+        for path in (F.PATH_AUTO, F.PATH_SIMT):
+            assert np.allclose(_run(q, k, v, F.BF16, scale, path), O.decode_attention(q, k, v, scale), rtol=RTOL, atol=ATOL)
 
 
 def test_over_the_compressed_cache_of_a_layer():
