@@ -1,17 +1,19 @@
 // Decode-step attention over a KV cache (Eq. 4) on the tensor cores, for bf16 caches with head_dim 128.
 //
 // One CTA takes a range of up to 15 tiles of 128 keys of one (unit, KV head) and all query heads of
-// the group (up to 16, zero-padded).  Both contractions run with the keys on the wide side, so the
+// the group (up to 8, zero-padded to the 16 rows of the narrow operand).  Both contractions run with the keys on the wide side, so the
 // tiny query side costs nothing and every K and V row is read from HBM exactly once:
 //   phase 1   S_t[key, head] = K_t Q^T        tcgen05.mma M = 128 keys, N = 16, contraction over head_dim;
 //             every tile's logits stay in TMEM (16 columns per tile)
 //   reduce    the exact per-head maximum over the CTA's range, from TMEM
-//   phase 2   P_t = 2^(c S_t - max) as bf16 into shared memory, then O[dim, head] += V_t^T P_t^T:
-//             M = 128 dims, N = 16, contraction over the tile's keys.  The V tile is the same swizzled
+//   phase 2   P_t = 2^(c S_t - max) into shared memory as two bf16 rows per head (the rounded weight and
+//             the rounding remainder), then O[dim, row] += V_t^T P_t^T: M = 128 dims, N = 16 = 8 heads x 2,
+//             contraction over the tile's keys; a head's output is the sum of its two columns.  The V tile is the same swizzled
 //             shared-memory tile a K tile is, read the other way round (MN-major operand), so V needs no
 //             transposition.  O never needs rescaling because the maximum is already final.
-// The CTA writes its unnormalised output, its maximum and its sum of weights; the join kernel of the
-// SIMT path (decode_combine_kernel) merges the ranges.
+// A head with one range is normalised and written at once.  Otherwise the CTA writes its unnormalised
+// output, its maximum and its sum of weights, and whichever range of a head finishes last (a ticket per
+// head) joins them all; the records it reads are L2-resident.
 // Roles: warp 0 lane 0 streams K tiles then V tiles through a three-stage TMA ring, warp 1 lane 0 issues
 // the MMAs, warps 2-5 (one thread per key of a tile / per output dim) do the softmax and the output.
 // Two CTAs fit an SM (256 TMEM columns, about 109 KB of shared memory each), so one streams while the
@@ -29,21 +31,24 @@ constexpr int kHeads = 16;                  // N of both contractions
 constexpr int kMaxHeads = 8;                // query heads per KV head this kernel serves
 constexpr int kMaxTiles = 15;               // 16 TMEM columns for O + 16 per score tile = 256
 constexpr int kTmemCols = 256;
+constexpr int kMaxJoin = 8192;               // (range, head) records the joining CTA can stage: ranges per head x heads
 constexpr int kThreads = 192;
 constexpr uint32_t kStageBytes = kTile * 128 * 2;            // both 64-element panels of a 128-row tile
 constexpr uint32_t kPanel = kStageBytes / 2;
 constexpr uint32_t kSmallPanel = kHeads * 128;               // 16 rows x 128 bytes
 constexpr uint32_t kSmemQ = kStages * kStageBytes;           // Q operand: two panels of 16 rows
 constexpr uint32_t kSmemP = kSmemQ + 2 * kSmallPanel;        // two P buffers of the same shape
-constexpr uint32_t kSmemRed = kSmemP + 4 * kSmallPanel;      // float [4 warps][8 heads]
+constexpr uint32_t kSmemRed = kSmemP + 4 * kSmallPanel;      // float [4 warps][8 heads], then the last-range flag
 constexpr uint32_t kSmemBar = kSmemRed + 256;
-constexpr int kBarFull = 0, kBarEmpty = kStages, kBarQ = 2 * kStages, kBarS = kBarQ + 1, kBarPFull = kBarS + 1,
-              kBarPEmpty = kBarPFull + 2, kBarO = kBarPEmpty + 2, kNumBars = kBarO + 1;
+constexpr int kBarFull = 0, kBarEmpty = kStages, kBarQ = 2 * kStages, kBarS = kBarQ + 1 /* one per score tile */,
+              kBarPFull = kBarS + kMaxTiles, kBarPEmpty = kBarPFull + 2, kBarO = kBarPEmpty + 2, kNumBars = kBarO + 1;
 constexpr uint32_t kSmemBytes = kSmemBar + 8 * kNumBars + 16;
 
 struct Args {
     const __nv_bfloat16 *q;     // [U, Hq, 128] dense
     float *part;                // [UH, n_split, G, 130]: unnormalised output, maximum (log2 domain), sum of weights
+    float *out;                 // [U, Hq, 128]
+    int *tickets;               // [UH], zero on entry and on exit: how many ranges of the head have finished
     int *status;
     int Hq, Hkv, G, N, n_split, tiles_per_split;
     float scale_log2;
@@ -135,8 +140,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
                     tc::umma_bf16(tmem + kHeads + kHeads * t, tc::smem_desc_sw128(a + (j >> 2) * kPanel, (j & 3) * 32),
                                   tc::smem_desc_sw128(base + kSmemQ + (j >> 2) * kSmallPanel, (j & 3) * 32), kIdescQK, j > 0);
                 tc::umma_commit(bar(kBarEmpty + st));
+                tc::umma_commit(bar(kBarS + t));
             }
-            if (ok) tc::umma_commit(bar(kBarS));
             for (int t = 0; ok && t < nt; ++t) {
                 const int i = nt + t, st = i % kStages, pb = t & 1;
                 ok = tc::mbar_wait(bar(kBarFull + st), (i / kStages) & 1, abort_flag, A.status) &&
@@ -169,12 +174,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
         fence_proxy_async();
         tc::mbar_arrive(bar(kBarQ));
 
-        bool ok = tc::mbar_wait(bar(kBarS), 0, abort_flag, A.status);
-        tc::tc_fence_after();
+        bool ok = true;
         float mx[kMaxHeads];
 #pragma unroll
         for (int g = 0; g < kMaxHeads; ++g) mx[g] = kNegBig;
-        for (int t = 0; t < nt; ++t) {
+        for (int t = 0; t < nt; ++t) {                               // running maxima while the K tiles stream
+            ok = ok && tc::mbar_wait(bar(kBarS + t), 0, abort_flag, A.status);
+            tc::tc_fence_after();
             uint32_t r[16];
             tc::tmem_ld16(trow + kHeads + kHeads * t, r);
             tc::tmem_ld_wait(r);
@@ -211,9 +217,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
             for (int g = 0; g < kMaxHeads; ++g) {
                 if (g < G) {
                     const float p = valid ? tc::ex2(fmaf(__uint_as_float(r[g]), A.scale_log2, -mref[g])) : 0.f;
-                    const __nv_bfloat16 pbf = __float2bfloat16_rn(p);
-                    l[g] += __bfloat162float(pbf);                   // the sum of the weights as the tensor core sees them
-                    sts16(prow + g * 128 + ((chunk ^ (g & 7)) << 4), __bfloat16_as_ushort(pbf));
+                    // bf16 head and bf16 remainder in rows g and 8 + g: their two products add up in fp32, so the
+                    // weight enters the second contraction with about 16 bits of mantissa
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(p), lo = __float2bfloat16_rn(p - __bfloat162float(hi));
+                    l[g] += p;
+                    const uint32_t at = prow + g * 128 + ((chunk ^ g) << 4);
+                    sts16(at, __bfloat16_as_ushort(hi));
+                    sts16(at + 1024, __bfloat16_as_ushort(lo));
                 }
             }
             fence_proxy_async();
@@ -228,20 +238,69 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
         epi_sync();
         ok = ok && tc::mbar_wait(bar(kBarO), 0, abort_flag, A.status);
         tc::tc_fence_after();
-        if (ok) {
-            uint32_t r[16];
-            tc::tmem_ld16(trow, r);
-            tc::tmem_ld_wait(r);
+        uint32_t r[16];
+        tc::tmem_ld16(trow, r);
+        tc::tmem_ld_wait(r);
+        float *out = A.out + ((int64_t)u * A.Hq + h * G) * 128 + row;
+        if (A.n_split == 1) {                                        // the only range of its head: normalise and finish
+#pragma unroll
+            for (int g = 0; g < kMaxHeads; ++g)
+                if (g < G && ok)
+                    out[g * 128] = (__uint_as_float(r[g]) + __uint_as_float(r[kMaxHeads + g])) /
+                                   (red[g] + red[kMaxHeads + g] + red[2 * kMaxHeads + g] + red[3 * kMaxHeads + g]);
+        } else {
             float *dst = A.part + ((int64_t)uh * A.n_split + split) * G * 130;
 #pragma unroll
-            for (int g = 0; g < kMaxHeads; ++g)
-                if (g < G) dst[g * 130 + row] = __uint_as_float(r[g]);
-#pragma unroll
-            for (int g = 0; g < kMaxHeads; ++g)
+            for (int g = 0; g < kMaxHeads; ++g) {
+                if (g < G) dst[g * 130 + row] = __uint_as_float(r[g]) + __uint_as_float(r[kMaxHeads + g]);
                 if (e == g && g < G) {
                     dst[g * 130 + 128] = mref[g];
                     dst[g * 130 + 129] = red[g] + red[kMaxHeads + g] + red[2 * kMaxHeads + g] + red[3 * kMaxHeads + g];
                 }
+            }
+            // the range that finishes last joins all ranges of its head
+            __threadfence();
+            epi_sync();
+            int *last = reinterpret_cast<int *>(red + 4 * kMaxHeads);
+            if (e == 0) {
+                const int done = atomicAdd(A.tickets + uh, 1);
+                *last = done == A.n_split - 1;
+                if (*last) A.tickets[uh] = 0;                        // ready for the next call
+            }
+            epi_sync();
+            if (*last && *abort_flag == 0) {        // both the same for all 128 threads: the barrier below is safe
+                __threadfence();
+                // maxima and sums of every (range, head) go through shared memory (the tile stages are idle by
+                // now), so that the long loop below is over independent loads only
+                const float *rec0 = A.part + (int64_t)uh * A.n_split * G * 130;
+                float *sm_m = reinterpret_cast<float *>(dtc_smem), *sm_l = sm_m + kMaxJoin;
+                const int n_rec = A.n_split * G;
+                for (int i = e; i < n_rec; i += 128) {
+                    sm_m[i] = __ldcg(rec0 + (int64_t)i * 130 + 128);
+                    sm_l[i] = __ldcg(rec0 + (int64_t)i * 130 + 129);
+                }
+                epi_sync();
+                float m[kMaxHeads], o[kMaxHeads], ls[kMaxHeads];
+#pragma unroll
+                for (int g = 0; g < kMaxHeads; ++g) {
+                    m[g] = kNegBig; o[g] = 0.f; ls[g] = 0.f;
+                    if (g < G)
+                        for (int sp = 0; sp < A.n_split; ++sp) m[g] = fmaxf(m[g], sm_m[sp * G + g]);
+                }
+#pragma unroll 2
+                for (int sp = 0; sp < A.n_split; ++sp) {             // all heads of two ranges in flight at a time
+#pragma unroll
+                    for (int g = 0; g < kMaxHeads; ++g)
+                        if (g < G) {
+                            const float w = tc::ex2(sm_m[sp * G + g] - m[g]);
+                            o[g] = fmaf(__ldcg(rec0 + ((int64_t)sp * G + g) * 130 + row), w, o[g]);
+                            ls[g] = fmaf(sm_l[sp * G + g], w, ls[g]);
+                        }
+                }
+#pragma unroll
+                for (int g = 0; g < kMaxHeads; ++g)
+                    if (g < G) out[g * 128] = o[g] / ls[g];
+            }
         }
     }
     tc::tc_fence_before();

@@ -622,11 +622,12 @@ flowmm_status validate_decode(const flowmm_decode_params *p) {
     return FLOWMM_OK;
 }
 
-// How a call is cut into key ranges, and where its scratch lives: [status word, 256 bytes][partial records].
+// How a call is cut into key ranges, and where its scratch lives:
+// [status word, 256 bytes][one ticket per (unit, KV head)][partial records].
 struct DecodePlan {
     bool tc;                 // tensor-core kernel (bf16, head_dim 128) or the SIMT one
     int n_split, per_split;  // ranges per (unit, KV head); keys (SIMT) or 128-key tiles (tensor core) per range
-    size_t bytes;
+    size_t part_off, bytes;
 };
 
 DecodePlan decode_plan(const flowmm_decode_params &p) {
@@ -634,13 +635,22 @@ DecodePlan decode_plan(const flowmm_decode_params &p) {
     const int uh = p.n_units * p.n_kv_heads, g = p.n_q_heads / p.n_kv_heads;
     d.tc = p.dtype == FLOWMM_BF16 && p.head_dim == 128 && p.path != FLOWMM_PATH_SIMT;
     if (d.tc) {
-        // two CTAs per SM; about two rounds of them when the cache is long enough, never more tiles than TMEM holds
+        // Two CTAs share an SM.  Of the range lengths TMEM allows, take the one with the least work per CTA
+        // slot when the CTAs run in rounds; a CTA's fixed cost (set-up, the pause between its two phases)
+        // counts like a tile and a half.
         const int tiles = (p.n_keys + dtc::kTile - 1) / dtc::kTile;
-        int per = (int)(((int64_t)tiles * uh + 4 * tc::sm_count() - 1) / (4 * tc::sm_count()));
-        per = per < 1 ? 1 : (per > dtc::kMaxTiles ? dtc::kMaxTiles : per);
-        d.per_split = per;
-        d.n_split = (tiles + per - 1) / per;
-    } else {
+        const int64_t slots = 2 * (int64_t)tc::sm_count();
+        double best = 0.0;
+        d.per_split = 1;
+        for (int per = 1; per <= dtc::kMaxTiles && per <= tiles; ++per) {
+            const int64_t ctas = (int64_t)uh * ((tiles + per - 1) / per);
+            const double cost = (double)((ctas + slots - 1) / slots) * (per + 1.5);
+            if (per == 1 || cost < best) { best = cost; d.per_split = per; }
+        }
+        d.n_split = (tiles + d.per_split - 1) / d.per_split;
+        if ((int64_t)d.n_split * g > dtc::kMaxJoin) d.tc = false;      // more ranges than the joining CTA can stage
+    }
+    if (!d.tc) {
         // enough CTAs for about four per SM, at least 64 keys each
         int want = (4 * 148 + uh - 1) / uh;
         const int max_split = (p.n_keys + 63) / 64;
@@ -648,7 +658,8 @@ DecodePlan decode_plan(const flowmm_decode_params &p) {
         d.per_split = (p.n_keys + want - 1) / want;
         d.n_split = (p.n_keys + d.per_split - 1) / d.per_split;
     }
-    d.bytes = 256 + align256((size_t)uh * d.n_split * g * (p.head_dim + 2) * sizeof(float));
+    d.part_off = 256 + align256((size_t)uh * sizeof(int));
+    d.bytes = d.part_off + align256((size_t)uh * d.n_split * g * (p.head_dim + 2) * sizeof(float));
     return d;
 }
 
@@ -670,8 +681,7 @@ flowmm_status launch_decode(const DecodeArgs &a, int uh, int n_q, cudaStream_t s
     return FLOWMM_OK;
 }
 
-flowmm_status launch_decode_tc(const flowmm_decode_params &p, const DecodeArgs &a, int *status, int uh, int n_q,
-                               cudaStream_t st) {
+flowmm_status launch_decode_tc(const flowmm_decode_params &p, const DecodeArgs &a, int *status, int uh, cudaStream_t st) {
     CUtensorMap kmap, vmap;
     const uint64_t dims[4] = {128, (uint64_t)p.n_keys, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
     const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
@@ -689,13 +699,12 @@ flowmm_status launch_decode_tc(const flowmm_decode_params &p, const DecodeArgs &
         configured = true;
     }
     dtc::Args t;
-    t.q = static_cast<const __nv_bfloat16 *>(a.q); t.part = a.part; t.status = status;
+    t.q = static_cast<const __nv_bfloat16 *>(a.q); t.part = a.part; t.out = a.out; t.status = status;
+    t.tickets = status + 64;
     t.Hq = a.Hq; t.Hkv = a.Hkv; t.G = a.G; t.N = a.N; t.n_split = a.n_split; t.tiles_per_split = a.keys_per_split;
     t.scale_log2 = a.scale_log2;
     dtc::decode_tc_kernel<<<dim3(a.n_split, uh), dtc::kThreads, dtc::kSmemBytes, st>>>(kmap, vmap, t);
     FLOWMM_LAUNCHED("decode_tc");
-    decode_combine_kernel<128><<<n_q, 128, 0, st>>>(a);
-    FLOWMM_LAUNCHED("decode_combine");
     return FLOWMM_OK;
 }
 
@@ -721,16 +730,16 @@ extern "C" flowmm_status flowmm_decode_attention(const flowmm_decode_params *p, 
     const DecodePlan plan = decode_plan(*p);
     if (ws_bytes < plan.bytes) return FLOWMM_ERR_WORKSPACE;
     FLOWMM_TRY(check_device());
-    if (cudaMemsetAsync(ws, 0, 4, st) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, plan.part_off, st) != cudaSuccess) return FLOWMM_ERR_CUDA;   // status word and tickets
     DecodeArgs a;
-    a.q = q; a.k = k; a.v = v; a.part = reinterpret_cast<float *>(static_cast<char *>(ws) + 256); a.out = out;
+    a.q = q; a.k = k; a.v = v; a.part = reinterpret_cast<float *>(static_cast<char *>(ws) + plan.part_off); a.out = out;
     a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads; a.G = p->n_q_heads / p->n_kv_heads; a.N = p->n_keys;
     a.n_split = plan.n_split; a.keys_per_split = plan.per_split;
     const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.f / sqrtf((float)p->head_dim);
     a.scale_log2 = scale * kLog2e;
     for (int i = 0; i < 3; ++i) { a.ks[i] = p->k_stride[i]; a.vs[i] = p->v_stride[i]; }
     const int uh = p->n_units * p->n_kv_heads, n_q = p->n_units * p->n_q_heads;
-    if (plan.tc) return launch_decode_tc(*p, a, static_cast<int *>(ws), uh, n_q, st);
+    if (plan.tc) return launch_decode_tc(*p, a, static_cast<int *>(ws), uh, st);
     if (p->dtype == FLOWMM_BF16)
         return p->head_dim == 128 ? launch_decode<__nv_bfloat16, 128>(a, uh, n_q, st) : launch_decode<__nv_bfloat16, 64>(a, uh, n_q, st);
     return p->head_dim == 128 ? launch_decode<float, 128>(a, uh, n_q, st) : launch_decode<float, 64>(a, uh, n_q, st);
