@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--path", default="auto", choices=["auto", "simt"])
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets held on the device (0 = automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="skip the decode-attention timing over the caches")
     ap.add_argument("--cpu-baseline-units", type=int, default=0)
     return ap.parse_args()
 
@@ -377,6 +378,43 @@ def run_ours(args):
     e2e_ms = shard.max_over_ranks(e2e_ms, dev)
     e2e_value = shard.aggregate_throughput(tokens_layers, world, e2e_ms / e2e_steps)
 
+    # the step this path feeds (not part of the timed metric): one decode query per head over every layer's
+    # cache, full length against compressed; L2 flushed before every call, each call timed on its own
+    decode = None
+    if not args.no_decode:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        comp = []
+        for q, k, v, m in sets:
+            ko, vo = torch.empty_like(k_out), torch.empty_like(v_out)
+            F.flowmm_compress_layer(p, q, k, v, m, ko, vo, ws)
+            comp.append((ko, vo))
+        q_dec = [t[0][:, :, -1, :].contiguous() for t in sets]
+        out_dec = torch.empty(q_dec[0].shape, dtype=torch.float32, device=dev)
+        decode = {}
+        for label, caches in (("full", [(t[1], t[2]) for t in sets]), ("compressed", comp)):
+            ws_d = torch.empty(F.flowmm_decode_workspace_bytes(q_dec[0], *caches[0]), dtype=torch.uint8, device=dev)
+            times = []
+            for i in range(3 + 10):
+                kk, vv = caches[i % n_sets]
+                flush.zero_()
+                e0.record()
+                F.flowmm_decode_attention(q_dec[i % n_sets], kk, vv, out_dec, ws_d)
+                e1.record()
+                torch.cuda.synchronize()
+                if i >= 3:
+                    times.append(e0.elapsed_time(e1))
+            status = F.flowmm_last_device_status(ws_d)
+            if status != 0:
+                raise RuntimeError("device status (decode): " + F.status_string(status))
+            ms = sorted(times)[len(times) // 2]
+            nbytes = 2 * caches[0][0].numel() * dsize
+            decode[label] = {"n_keys": caches[0][0].shape[2], "ms": round(ms, 5), "bytes": nbytes,
+                             "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                             "frac_hbm": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+        decode["speedup"] = round(decode["full"]["ms"] / decode["compressed"]["ms"], 3)
+        decode["what"] = "flowmm_decode_attention, one query per head, all %d units in one call, per GPU" % U
+        del comp, flush
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -396,6 +434,8 @@ def run_ours(args):
             "kernels": {n: {k2: (round(v2, 5) if isinstance(v2, float) else v2) for k2, v2 in d.items()}
                         for n, d in kernels.items()},
         }
+        if decode is not None:
+            line["decode"] = decode
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl, args.permille, args.cpu_baseline_units)
         print(json.dumps(line))

@@ -67,7 +67,11 @@ typedef enum { FLOWMM_MERGE_EXPSIM = 0, FLOWMM_MERGE_MEAN = 1 } flowmm_merge_mod
 /* ABS: tau is compared with the importance directly.  REL: tau is in units of the
  * importance a uniform attention would give, tau_eff = tau * W / L. */
 typedef enum { FLOWMM_TAU_ABS = 0, FLOWMM_TAU_REL = 1 } flowmm_tau_mode;
-typedef enum { FLOWMM_FLOW_AUTO = 0, FLOWMM_FLOW_FORCE_INTRA = 1, FLOWMM_FLOW_FORCE_CROSS = 2 } flowmm_flow_mode;
+/* AUTO: the theta rule on rho (aligned merging).  FORCE_*: one strategy for every layer.  MISALIGNED: the
+ * reverse of the rule (intra-modal where rho > theta, cross-modal elsewhere), the contrast case of the paper's
+ * study of flow-aligned merging. */
+typedef enum { FLOWMM_FLOW_AUTO = 0, FLOWMM_FLOW_FORCE_INTRA = 1, FLOWMM_FLOW_FORCE_CROSS = 2,
+               FLOWMM_FLOW_MISALIGNED = 3 } flowmm_flow_mode;
 /* Which kernels do the two dense contractions.  AUTO: tensor-core (tcgen05) kernels when
  * dtype is bf16 and head_dim is 128, SIMT fp32 kernels otherwise.  SIMT forces the latter. */
 typedef enum { FLOWMM_PATH_AUTO = 0, FLOWMM_PATH_SIMT = 1 } flowmm_path;

@@ -51,7 +51,7 @@ typedef struct {
     double softmax_scale;   /* 0 -> 1/sqrt(head_dim) */
     double theta, tau;
     int32_t tau_mode;       /* 0 absolute, 1 relative: tau_eff = tau * W / L */
-    int32_t flow_mode;      /* 0 auto, 1 force intra, 2 force cross */
+    int32_t flow_mode;      /* 0 auto, 1 force intra, 2 force cross, 3 misaligned (the reverse of auto) */
     int32_t merge_mode;     /* 0 exp-similarity weights, 1 uniform mean */
     int32_t keep_window;    /* 1: the last W tokens are always pivots */
 } oracle_params;
@@ -146,6 +146,7 @@ int flowmm_oracle_layer_flow(const oracle_params *p, const double *cross, const 
         rho[u] = s / (double)Hq;
         if (p->flow_mode == 1) strategy[u] = 0;
         else if (p->flow_mode == 2) strategy[u] = 1;
+        else if (p->flow_mode == 3) strategy[u] = rho[u] > p->theta ? 0 : 1;   /* the misaligned contrast of the flow-merging study */
         else strategy[u] = rho[u] > p->theta ? 1 : 0;
     }
     return 0;

@@ -33,7 +33,7 @@ class _Params(ctypes.Structure):
 
 
 TAU_ABS, TAU_REL = 0, 1
-FLOW_AUTO, FLOW_FORCE_INTRA, FLOW_FORCE_CROSS = 0, 1, 2
+FLOW_AUTO, FLOW_FORCE_INTRA, FLOW_FORCE_CROSS, FLOW_MISALIGNED = 0, 1, 2, 3
 MERGE_EXPSIM, MERGE_MEAN = 0, 1
 INTRA, CROSS = 0, 1
 

@@ -159,7 +159,7 @@ flowmm_status validate(const flowmm_params *p) {
     if (p->n_keep < 1 || p->n_keep > p->seq_len) return FLOWMM_ERR_BUDGET;
     if (p->keep_window && p->n_keep < p->window) return FLOWMM_ERR_BUDGET;
     if (p->dtype != FLOWMM_F32 && p->dtype != FLOWMM_BF16) return FLOWMM_ERR_DTYPE;
-    if (p->tau_mode < 0 || p->tau_mode > 1 || p->flow_mode < 0 || p->flow_mode > 2 || p->merge_mode < 0 ||
+    if (p->tau_mode < 0 || p->tau_mode > 1 || p->flow_mode < 0 || p->flow_mode > 3 || p->merge_mode < 0 ||
         p->merge_mode > 1 || p->path < 0 || p->path > 1)
         return FLOWMM_ERR_SHAPE;
     if (!(p->softmax_scale >= 0.f) || isnan(p->theta) || isnan(p->tau)) return FLOWMM_ERR_SHAPE;

@@ -263,7 +263,7 @@ __global__ void layer_flow_kernel(const float *cross_mass, int U, int Hq, int W,
     for (int g = 0; g < Hq; ++g) s += cross_mass[(int64_t)u * Hq + g] / (float)W;   // a head's total mass is W
     const float r = s / (float)Hq;
     if (rho) rho[u] = r;
-    strategy[u] = flow_mode == 1 ? 0 : flow_mode == 2 ? 1 : (r > theta ? 1 : 0);
+    strategy[u] = flow_mode == 1 ? 0 : flow_mode == 2 ? 1 : ((r > theta) != (flow_mode == 3) ? 1 : 0);
 }
 
 // cross_mass_reduce and layer_flow_kernel in one launch (same sums in the same order): one block
@@ -282,7 +282,7 @@ __global__ void flow_from_parts_kernel(const float *cross_part, int n_chunk, int
         for (int g = 0; g < Hq; ++g) s += cross_mass[(int64_t)u * Hq + g] / (float)W;   // a head's total mass is W
         const float r = s / (float)Hq;
         if (rho) rho[u] = r;
-        strategy[u] = flow_mode == 1 ? 0 : flow_mode == 2 ? 1 : (r > theta ? 1 : 0);
+        strategy[u] = flow_mode == 1 ? 0 : flow_mode == 2 ? 1 : ((r > theta) != (flow_mode == 3) ? 1 : 0);
     }
 }
 

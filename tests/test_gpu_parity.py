@@ -45,11 +45,13 @@ def test_cfg4_video_mixed_window(permille):
     _check(configs.get("cfg4"), [(2, 0), (20, 0)], permille)
 
 
-@pytest.mark.parametrize("mode", ["mean", "force_intra", "force_cross", "no_gate", "keep_window", "abs_tau"])
+@pytest.mark.parametrize("mode", ["mean", "force_intra", "force_cross", "misaligned", "no_flow_no_gate", "no_gate",
+                                  "keep_window", "abs_tau"])
 def test_variants(mode):
     wl = configs.get("cfg2")
     kw = {"mean": dict(merge_mode=O.MERGE_MEAN), "force_intra": dict(flow_mode=O.FLOW_FORCE_INTRA),
-          "force_cross": dict(flow_mode=O.FLOW_FORCE_CROSS), "no_gate": dict(tau=float("inf")),
+          "force_cross": dict(flow_mode=O.FLOW_FORCE_CROSS), "misaligned": dict(flow_mode=O.FLOW_MISALIGNED),
+          "no_flow_no_gate": dict(flow_mode=O.FLOW_FORCE_CROSS, tau=float("inf")), "no_gate": dict(tau=float("inf")),
           "keep_window": dict(keep_window=1), "abs_tau": dict(tau=0.3, tau_mode=O.TAU_ABS)}[mode]
     _check(wl, [(3, 0), (29, 0)], 100, **kw)
 

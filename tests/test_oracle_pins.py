@@ -139,6 +139,8 @@ def test_flow_threshold_rule():
     assert O.layer_flow(p, cross, total)[1].tolist() == [0, 0, 0]
     p.flow_mode = O.FLOW_FORCE_CROSS
     assert O.layer_flow(p, cross, total)[1].tolist() == [1, 1, 1]
+    p.flow_mode = O.FLOW_MISALIGNED                          # the reverse of the rule, layer by layer
+    assert O.layer_flow(p, cross, total)[1].tolist() == [O.CROSS, O.INTRA, O.INTRA]
     # head mean of ratios, not ratio of sums
     rho2, _ = O.layer_flow(params(U=1, Hq=2), np.array([[1.0, 0.0]]), np.array([[2.0, 8.0]]))
     assert abs(rho2[0] - 0.25) < 1e-15
