@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "decode.cuh"
 #include "decode_tc.cuh"
+#include "merge_tc.cuh"
 #include "match_tc.cuh"
 #include "score_tc.cuh"
 #include "select_merge.cuh"
@@ -59,6 +60,8 @@ struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
     size_t row_part, cross_part, rn, sort_a, sort_b, mem_tok, mem_w, piece_desc, off, piece_off, part_off, partial, ticket, slot_done;
     size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod, negc;
+    size_t tokmap;             // [UH, L] (slot, weight) of every token position, for the tensor-core merge
+    size_t merge_status;       // status word the merge kernels report to (the workspace's own, or one of the merge scratch)
     int tc_n_qt, tc_n_chunk, tc_tiles_per_chunk, gw_pad;
     size_t total;
     int n_chunk1, chunk1, n_chunk2, chunk2, max_pieces, max_parts, csr_passes, c_tot, n_rt;
@@ -93,6 +96,8 @@ void layout_merge(Layout &y, const flowmm_params &p, Take take) {
     y.partial = take(UH * (size_t)y.max_parts * (2 * D + 4) * 4);
     y.ticket = take(256);
     y.slot_done = take(UH * B * 4);
+    y.merge_status = take(256);
+    y.tokmap = take(UH * (size_t)p.seq_len * 8);
 }
 
 Layout make_layout(const flowmm_params &p) {
@@ -138,6 +143,7 @@ Layout make_layout(const flowmm_params &p) {
     y.negc = take(U * Hkv * (size_t)y.gw_pad * 4);
     y.rn = take(U * Hkv * L * 4);
     layout_merge(y, p, take);
+    y.merge_status = y.status;
     y.c_tot = (int)((B + 31) / 32 * 32 + 32);
     y.cand_k = take(U * Hkv * (size_t)y.c_tot * 128 * 2);
     y.cand_scale = take(U * Hkv * (size_t)y.c_tot * 4 + 1024);   // + one tile of slack: whole 256-column slices are copied
@@ -402,6 +408,34 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
     m.max_pieces = E == 0 ? p.n_keep : y.max_pieces; m.max_parts = y.max_parts;
     for (int i = 0; i < 3; ++i) {
         m.ks[i] = p.k_stride[i]; m.vs[i] = p.v_stride[i]; m.kos[i] = p.ko_stride[i]; m.vos[i] = p.vo_stride[i];
+    }
+    // few slots per head: Eq. 5 as a product with the slot-by-token weight matrix on the tensor cores
+    if (E > 0 && p.dtype == FLOWMM_BF16 && p.head_dim == 128 && p.n_keep <= mtc::kMaxSlots && p.seq_len < 65536 &&
+        p.path != FLOWMM_PATH_SIMT) {       // (below 65536 tokens a slot's fixed-point weight sum cannot overflow)
+        mtc::MapArgs ma;
+        ma.retained = retained; ma.evicted = evicted; ma.match = match; ma.match_sim = match_sim;
+        ma.tokmap = at<int2>(ws, y.tokmap); ma.L = p.seq_len; ma.B = p.n_keep; ma.E = E; ma.merge_mode = p.merge_mode;
+        const int longest = E > p.n_keep ? E : p.n_keep;
+        mtc::merge_map_kernel<<<dim3((longest + 255) / 256, UH), 256, 0, st>>>(ma);
+        FLOWMM_LAUNCHED("merge_map");
+        CUtensorMap kmap, vmap;
+        const uint64_t dims[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
+        const uint64_t ksb[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
+        const uint64_t vsb[3] = {(uint64_t)p.v_stride[2] * 2, (uint64_t)p.v_stride[1] * 2, (uint64_t)p.v_stride[0] * 2};
+        const uint32_t box[4] = {64, mtc::kTile, 1, 1};
+        if (!tc::make_bf16_map(&kmap, k, 4, dims, ksb, box) || !tc::make_bf16_map(&vmap, v, 4, dims, vsb, box))
+            return FLOWMM_ERR_CUDA;
+        mtc::Args a;
+        a.tokmap = ma.tokmap; a.k_out = k_out; a.v_out = v_out; a.status = at<int>(ws, y.merge_status);
+        a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.B = p.n_keep; a.n_items = UH; a.n_stages = mtc::kMaxStages;
+        for (int i = 0; i < 3; ++i) { a.kos[i] = p.ko_stride[i]; a.vos[i] = p.vo_stride[i]; }
+        const uint32_t smem = mtc::smem_bytes(p.n_keep, a.n_stages);
+        if (cudaFuncSetAttribute(mtc::merge_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return FLOWMM_ERR_CUDA;
+        const int grid = UH < tc::sm_count() ? UH : tc::sm_count();
+        mtc::merge_tc_kernel<<<grid, mtc::kThreads, smem, st>>>(kmap, vmap, a);
+        FLOWMM_LAUNCHED("merge_tc");
+        return FLOWMM_OK;
     }
     if (E > 0) {
         CsrArgs c;
