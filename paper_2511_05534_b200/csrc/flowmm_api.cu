@@ -12,6 +12,7 @@
 #include "decode.cuh"
 #include "decode_tc.cuh"
 #include "merge_tc.cuh"
+#include "score_fused_tc.cuh"
 #include "match_tc.cuh"
 #include "score_tc.cuh"
 #include "select_merge.cuh"
@@ -263,8 +264,54 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     return FLOWMM_OK;
 }
 
+// Short contexts with few proxy rows per KV head: every logit of a head fits in TMEM, K is read once.
+bool use_fused_score(const flowmm_params &p) {
+    const int gw = p.n_q_heads / p.n_kv_heads * p.window, nt = (p.seq_len + sft::kTile - 1) / sft::kTile;
+    return use_tc(p) && (gw == 32 || gw == 64) && nt <= sft::kMaxTiles && nt * gw <= 512 &&
+           p.window <= 256 && p.n_q_heads / p.n_kv_heads <= 256;
+}
+
+template <int GW>
+flowmm_status launch_score_fused(const CUtensorMap &qmap, const CUtensorMap &kmap, const sft::Args &a, int uh,
+                                 cudaStream_t st) {
+    const uint32_t smem = sft::Smem<GW>::bytes((a.L + sft::kTile - 1) / sft::kTile);
+    if (cudaFuncSetAttribute(sft::score_fused_tc_kernel<GW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(sft::score_fused_tc_kernel<GW>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        return FLOWMM_ERR_CUDA;
+    sft::score_fused_tc_kernel<GW><<<uh, sft::kThreads, smem, st>>>(qmap, kmap, a);
+    FLOWMM_LAUNCHED("score_fused_tc");
+    return FLOWMM_OK;
+}
+
+flowmm_status run_score_fused(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
+                              float *importance, float *cross_mass, void *ws, cudaStream_t st) {
+    const int UH = p.n_units * p.n_kv_heads, G = p.n_q_heads / p.n_kv_heads, W = p.window, GW = G * W;
+    CUtensorMap qmap, kmap;
+    const uint64_t qd[4] = {128, (uint64_t)W, (uint64_t)p.n_q_heads, (uint64_t)p.n_units};
+    const uint64_t qs[3] = {(uint64_t)p.q_stride[2] * 2, (uint64_t)p.q_stride[1] * 2, (uint64_t)p.q_stride[0] * 2};
+    const uint64_t kd[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
+    const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
+    const uint32_t bq[4] = {64, (uint32_t)W, (uint32_t)G, 1}, bk[4] = {64, sft::kTile, 1, 1};
+    if (!tc::make_bf16_map(&qmap, q, 4, qd, qs, bq) || !tc::make_bf16_map(&kmap, k, 4, kd, ks, bk)) return FLOWMM_ERR_CUDA;
+    sft::Args a;
+    a.modality = mod; a.importance = importance; a.cross_mass = cross_mass; a.status = at<int>(ws, y.status);
+    a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.G = G; a.W = W; a.L = p.seq_len; a.GW = GW;
+    const int need = (p.seq_len + sft::kTile - 1) / sft::kTile * GW;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < need) a.tmem_cols *= 2;
+    const float scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * kLog2e;
+    return GW == 32 ? launch_score_fused<32>(qmap, kmap, a, UH, st) : launch_score_fused<64>(qmap, kmap, a, UH, st);
+}
+
+// parts_out: the caller reduces the partial cross-modal masses itself; set to 0 when cross_mass is already final
 flowmm_status run_score(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
                         float *importance, float *cross_mass, void *ws, cudaStream_t st, int *parts_out = nullptr) {
+    if (use_fused_score(p)) {
+        if (parts_out) *parts_out = 0;
+        return run_score_fused(p, y, q, k, mod, importance, cross_mass, ws, st);
+    }
     if (use_tc_score(p)) return run_score_tc(p, y, q, k, mod, importance, cross_mass, ws, st, parts_out);
     ScoreArgs a;
     a.q = q; a.k = k; a.modality = mod; a.importance = importance;
@@ -577,9 +624,13 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
     float *cross_mass = at<float>(ws, y.cross_mass);
     int n_parts = 0;
     FLOWMM_TRY(run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, st, &n_parts));
-    flow_from_parts_kernel<<<p->n_units, 256, 0, st>>>(at<float>(ws, y.cross_part), n_parts, p->n_q_heads, p->window,
-                                                       p->theta, p->flow_mode, cross_mass, rho, strategy);
-    FLOWMM_LAUNCHED("flow_from_parts");
+    if (n_parts == 0) {
+        FLOWMM_TRY(run_layer_flow(*p, cross_mass, rho, strategy, st));
+    } else {
+        flow_from_parts_kernel<<<p->n_units, 256, 0, st>>>(at<float>(ws, y.cross_part), n_parts, p->n_q_heads, p->window,
+                                                           p->theta, p->flow_mode, cross_mass, rho, strategy);
+        FLOWMM_LAUNCHED("flow_from_parts");
+    }
     FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st));
     FLOWMM_TRY(run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws, st));
     FLOWMM_TRY(run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws, st));

@@ -63,7 +63,7 @@ def test_errors_are_reported_not_computed():
         F.flowmm_score(fp, q, k_odd, m, imp, cross, ws)
     assert e.value.code == 6
     F.flowmm_score(fp, q, k, m, imp, cross, ws)
-    assert F.flowmm_last_launch_count() >= 2
+    assert F.flowmm_last_launch_count() >= 1
     torch.cuda.synchronize()
 
 
