@@ -264,29 +264,15 @@ flowmm_status run_score_tc(const flowmm_params &p, const Layout &y, const void *
     return FLOWMM_OK;
 }
 
-// Short contexts with few proxy rows per KV head: every logit of a head fits in TMEM, K is read once.
+// Short contexts with 32 proxy rows per KV head: every logit of a head fits in half of TMEM, K is read once.
 bool use_fused_score(const flowmm_params &p) {
     const int gw = p.n_q_heads / p.n_kv_heads * p.window, nt = (p.seq_len + sft::kTile - 1) / sft::kTile;
-    return use_tc(p) && (gw == 32 || gw == 64) && nt <= sft::kMaxTiles && nt * gw <= 512 &&
-           p.window <= 256 && p.n_q_heads / p.n_kv_heads <= 256;
-}
-
-template <int GW>
-flowmm_status launch_score_fused(const CUtensorMap &qmap, const CUtensorMap &kmap, const sft::Args &a, int uh,
-                                 cudaStream_t st) {
-    const uint32_t smem = sft::Smem<GW>::bytes((a.L + sft::kTile - 1) / sft::kTile);
-    if (cudaFuncSetAttribute(sft::score_fused_tc_kernel<GW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaFuncSetAttribute(sft::score_fused_tc_kernel<GW>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared) != cudaSuccess)
-        return FLOWMM_ERR_CUDA;
-    sft::score_fused_tc_kernel<GW><<<uh, sft::kThreads, smem, st>>>(qmap, kmap, a);
-    FLOWMM_LAUNCHED("score_fused_tc");
-    return FLOWMM_OK;
+    return use_tc(p) && gw == sft::kRows && nt <= sft::kMaxTiles;
 }
 
 flowmm_status run_score_fused(const flowmm_params &p, const Layout &y, const void *q, const void *k, const uint8_t *mod,
                               float *importance, float *cross_mass, void *ws, cudaStream_t st) {
-    const int UH = p.n_units * p.n_kv_heads, G = p.n_q_heads / p.n_kv_heads, W = p.window, GW = G * W;
+    const int UH = p.n_units * p.n_kv_heads, G = p.n_q_heads / p.n_kv_heads, W = p.window;
     CUtensorMap qmap, kmap;
     const uint64_t qd[4] = {128, (uint64_t)W, (uint64_t)p.n_q_heads, (uint64_t)p.n_units};
     const uint64_t qs[3] = {(uint64_t)p.q_stride[2] * 2, (uint64_t)p.q_stride[1] * 2, (uint64_t)p.q_stride[0] * 2};
@@ -296,13 +282,16 @@ flowmm_status run_score_fused(const flowmm_params &p, const Layout &y, const voi
     if (!tc::make_bf16_map(&qmap, q, 4, qd, qs, bq) || !tc::make_bf16_map(&kmap, k, 4, kd, ks, bk)) return FLOWMM_ERR_CUDA;
     sft::Args a;
     a.modality = mod; a.importance = importance; a.cross_mass = cross_mass; a.status = at<int>(ws, y.status);
-    a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.G = G; a.W = W; a.L = p.seq_len; a.GW = GW;
-    const int need = (p.seq_len + sft::kTile - 1) / sft::kTile * GW;
-    a.tmem_cols = 32;
-    while (a.tmem_cols < need) a.tmem_cols *= 2;
+    a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.G = G; a.W = W; a.L = p.seq_len; a.n_items = UH;
     const float scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * kLog2e;
-    return GW == 32 ? launch_score_fused<32>(qmap, kmap, a, UH, st) : launch_score_fused<64>(qmap, kmap, a, UH, st);
+    if (cudaFuncSetAttribute(sft::score_fused_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)sft::kSmemBytes) != cudaSuccess)
+        return FLOWMM_ERR_CUDA;
+    const int grid = UH < tc::sm_count() ? UH : tc::sm_count();
+    sft::score_fused_tc_kernel<<<grid, sft::kThreads, sft::kSmemBytes, st>>>(qmap, kmap, a);
+    FLOWMM_LAUNCHED("score_fused_tc");
+    return FLOWMM_OK;
 }
 
 // parts_out: the caller reduces the partial cross-modal masses itself; set to 0 when cross_mass is already final
