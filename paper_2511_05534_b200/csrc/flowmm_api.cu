@@ -463,7 +463,7 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
             return FLOWMM_ERR_CUDA;
         mtc::Args a;
         a.tokmap = ma.tokmap; a.k_out = k_out; a.v_out = v_out; a.status = at<int>(ws, y.merge_status);
-        a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.B = p.n_keep; a.n_items = UH; a.n_stages = mtc::kMaxStages;
+        a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.B = p.n_keep; a.n_items = UH; a.n_stages = p.n_keep <= 128 ? mtc::kMaxStages : 3;
         for (int i = 0; i < 3; ++i) { a.kos[i] = p.ko_stride[i]; a.vos[i] = p.vo_stride[i]; }
         const uint32_t smem = mtc::smem_bytes(p.n_keep, a.n_stages);
         if (cudaFuncSetAttribute(mtc::merge_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

@@ -1,4 +1,4 @@
-// Weighted merge (Eq. 5) + compaction on the tensor cores, for budgets of up to 128 pivots per head
+// Weighted merge (Eq. 5) + compaction on the tensor cores, for budgets of up to 240 pivots per head
 // (bf16, head_dim 128).
 //
 // Eq. 5 is out = W X with X the head's L rows of K (or V) and W a B x L matrix with one non-zero per
@@ -14,8 +14,8 @@
 //       over the step's tokens; the X tile is the swizzled TMA tile read as an MN-major operand, for K
 //       and for V against the same W slice;
 //       after the last step four reader warps take out^T from TMEM, scale by 1 / (1 + sum of weights)
-//       and store bf16 rows, while the next head's steps already run into a second set of accumulators
-//       and a second set of sums.
+//       and store bf16 rows, while the next head's steps already run into a second set of sums and (up to
+//       128 slots) a second set of accumulators.
 // The weights enter rounded to bf16 (relative error <= 2^-9) in numerator and denominator alike, so every
 // output row is still a weighted mean of its members with weights within 0.2 % of Eq. 5's; the change of
 // the result is below the bf16 rounding of the output itself.
@@ -31,7 +31,7 @@ namespace flowmm {
 namespace mtc {
 
 constexpr int kTile = 128;                       // tokens per step
-constexpr int kMaxSlots = 128;
+constexpr int kMaxSlots = 240;                   // N <= 240: two 60 KB weight slices and three tile stages fit in shared memory
 constexpr int kThreads = 320;                    // TMA warp, MMA warp, four builder warps, four reader warps
 constexpr int kPivotFlag = 1 << 30;              // in the table's slot word: the token is the slot's pivot
 constexpr uint32_t kStageBytes = kTile * 128 * 2, kPanel = kStageBytes / 2;
@@ -85,8 +85,9 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     extern __shared__ __align__(1024) uint8_t mtc_smem[];
     const uint32_t base = tc::smem_u32(mtc_smem);
     const int N = slots16(A.B);
-    constexpr int n_sets = 2;                                        // accumulator sets in TMEM: K at column 0, V at column 128 of a set
-    constexpr uint32_t set_cols = 256u, v_col = 128u;
+    // accumulator sets in TMEM: up to 128 slots two sets (K at column 0, V at column 128 of a set), else one (V at 256)
+    const int n_sets = N <= 128 ? 2 : 1;
+    const uint32_t set_cols = 256u, v_col = N <= 128 ? 128u : 256u;
     const uint32_t wsize = w_bytes(A.B), wpanel = (uint32_t)N * 128u;
     const uint32_t w0 = base + (uint32_t)A.n_stages * kStageBytes;
     uint8_t *tail = mtc_smem + (size_t)A.n_stages * kStageBytes + 2 * (size_t)wsize;
@@ -223,8 +224,10 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
             const int set = it % n_sets, use = it / n_sets;
             unsigned *sums = wsum + set * kMaxSlots;
             ok = ok && tc::mbar_wait(bar(kBarSumFull + set), use & 1, abort_flag, A.status);
-            inv_s[e] = 1.f / (1.f + (float)sums[e] * (1.f / kSumScale));
-            sums[e] = 0u;
+            for (int sl = e; sl < N; sl += 128) {
+                inv_s[sl] = 1.f / (1.f + (float)sums[sl] * (1.f / kSumScale));
+                sums[sl] = 0u;
+            }
             reader_sync();
             ok = ok && tc::mbar_wait(bar(kBarOutFull + set), use & 1, abort_flag, A.status);
             tc::tc_fence_after();
