@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "decode.cuh"
 #include "decode_tc.cuh"
+#include "match_small_tc.cuh"
 #include "merge_tc.cuh"
 #include "score_fused_tc.cuh"
 #include "match_tc.cuh"
@@ -378,6 +379,22 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     const uint64_t ks[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
     const uint64_t cd[4] = {128, (uint64_t)y.c_tot, (uint64_t)UH, 1};
     const uint64_t cs[3] = {256, (uint64_t)y.c_tot * 256, (uint64_t)y.c_tot * 256 * (uint64_t)UH};
+    if (y.c_tot <= mst::kMaxCols) {      // the whole candidate list of a head is one operand tile
+        const uint32_t box_t[4] = {64, mst::kTile, 1, 1}, box_c[4] = {64, (uint32_t)y.c_tot, 1, 1};
+        if (!tc::make_bf16_map(&k_map, k, 4, kd, ks, box_t) || !tc::make_bf16_map(&cand_map, g.cand_k, 4, cd, cs, box_c))
+            return FLOWMM_ERR_CUDA;
+        mst::Args a;
+        a.cand_count = g.cand_count; a.cand_slot = g.cand_slot; a.rank = g.rank; a.strategy = strategy;
+        a.cand_scale = g.cand_scale; a.modality = mod; a.match = match; a.match_sim = match_sim;
+        a.status = at<int>(ws, y.status);
+        a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.E = E; a.Ctot = y.c_tot; a.n_heads = UH;
+        if (cudaFuncSetAttribute(mst::match_small_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)mst::kSmemBytes) != cudaSuccess)
+            return FLOWMM_ERR_CUDA;
+        mst::match_small_tc_kernel<<<UH < tc::sm_count() ? UH : tc::sm_count(), mst::kThreads, mst::kSmemBytes, st>>>(k_map, cand_map, a);
+        FLOWMM_LAUNCHED("match_small_tc");
+        return FLOWMM_OK;
+    }
     // few candidates per head: the token rows are the stream, take the shape with two A stages
     const bool small = y.c_tot <= 128;
     const uint32_t box_a[4] = {64, kMtRows, 1, 1};
