@@ -1,12 +1,13 @@
-// Matching step (Eq. 9 and Eq. 10) on the tensor cores for short candidate lists (at most 128 columns
-// per head, i.e. budgets of up to 96 pivots): the whole candidate matrix of a head is one operand tile.
+// Matching step (Eq. 9 and Eq. 10) on the tensor cores for short candidate lists (at most 256 columns
+// per head, i.e. budgets of up to 224 pivots): the whole candidate matrix of a head is one operand tile.
 //
 // Same preparation as match_tc.cuh (match_prepare_kernel: admissible pivots gathered into a dense matrix,
 // text group first, visual group from the next multiple of 32, NaN scales where there is no candidate).
 // CTAs are persistent (one per SM) and take whole heads: warp 0 lane 0 loads the head's candidate tile,
-// its reciprocal norms and slots (double-buffered by head) and streams the head's 128-token tiles through
-// a TMA ring; warp 1 lane 0 issues S = K_tile C^T (tcgen05.mma, M = 128 tokens, N = candidates) into
-// one of four TMEM accumulators; four teams of four warps take the tiles in turn: a thread owns a token,
+// its reciprocal norms and slots (double-buffered by head up to 128 columns) and streams the head's
+// 128-token tiles through a TMA ring; warp 1 lane 0 issues S = K_tile C^T (tcgen05.mma, M = 128 tokens,
+// N = candidates) into one of four (two above 128 columns) TMEM accumulators; four teams of four warps
+// take the tiles in turn: a thread owns a token,
 // reads its key row from the A stage for the norm, walks its admissible candidate blocks (an intra-modal
 // layer: only the blocks of the token's own modality), keeps the running maximum per group of 8 columns
 // and recovers the exact column at the end.  Nothing is handed between warps.
@@ -20,18 +21,18 @@ namespace mst {
 
 constexpr int kTile = 128;
 constexpr int kStages = 4;
-constexpr int kMaxCols = 128;
-constexpr int kSets = 4;                      // TMEM accumulators of 128 columns
+constexpr int kMaxCols = 256;
+constexpr int kMaxSets = 4;                   // TMEM accumulators: four of 128 columns or two of 256
 constexpr int kTeams = 4;
 constexpr int kThreads = 64 + kTeams * 128;
 constexpr uint32_t kStageBytes = kTile * 128 * 2, kPanel = kStageBytes / 2;
-constexpr uint32_t kBBytes = kMaxCols * 256;                       // candidate tile of one head: two panels of N rows
-constexpr uint32_t kSmemB = kStages * kStageBytes;                 // two candidate tiles
-constexpr uint32_t kSmemMeta = kSmemB + 2 * kBBytes;               // per head buffer: float scale[128], int slot[128]
-constexpr uint32_t kSmemStash = kSmemMeta + 2 * 1024;              // per team: 8 floats per row
+constexpr uint32_t kBRegion = kMaxCols * 256;                      // candidate tiles (two panels of N rows each): two of up to 128 rows or one
+constexpr uint32_t kSmemB = kStages * kStageBytes;
+constexpr uint32_t kSmemMeta = kSmemB + kBRegion;                  // per candidate buffer: float scale[N], int slot[N]
+constexpr uint32_t kSmemStash = kSmemMeta + 4096;                  // per team: 8 floats per row
 constexpr uint32_t kSmemBar = kSmemStash + kTeams * 4096;
 constexpr int kBarFull = 0, kBarEmpty = kStages, kBarBFull = 2 * kStages, kBarBEmpty = kBarBFull + 2,
-              kBarAccFull = kBarBEmpty + 2, kBarSetFree = kBarAccFull + kSets, kNumBars = kBarSetFree + kSets;
+              kBarAccFull = kBarBEmpty + 2, kBarSetFree = kBarAccFull + kMaxSets, kNumBars = kBarSetFree + kMaxSets;
 constexpr uint32_t kSmemBytes = kSmemBar + 8 * kNumBars + 16;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
@@ -58,6 +59,8 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     }
     const int nt = (A.L + kTile - 1) / kTile, N = A.Ctot;
     const uint32_t b_bytes = (uint32_t)N * 256u, b_panel = (uint32_t)N * 128u;
+    const int n_sets = N <= 128 ? 4 : 2, n_bbuf = N <= 128 ? 2 : 1;
+    const uint32_t set_cols = N <= 128 ? 128u : 256u, b_stride = kBRegion / 2, m_stride = 2048, slot_off = 4u * (uint32_t)N;
     auto bar = [&](int i) { return bars + 8u * i; };
     if (threadIdx.x == 0) {
         for (int i = 0; i < kNumBars; ++i) {
@@ -83,15 +86,15 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             bool ok = true;
             int i = 0, hc = 0;
             for (int uh = blockIdx.x; ok && uh < A.n_heads; uh += gridDim.x, ++hc) {
-                const int u = uh / A.Hkv, h = uh % A.Hkv, hp = hc & 1;
-                ok = tc::mbar_wait(bar(kBarBEmpty + hp), ((hc >> 1) & 1) ^ 1, abort_flag, A.status);
+                const int u = uh / A.Hkv, h = uh % A.Hkv, hp = hc % n_bbuf;
+                ok = tc::mbar_wait(bar(kBarBEmpty + hp), ((hc / n_bbuf) & 1) ^ 1, abort_flag, A.status);
                 if (!ok) break;
-                const uint32_t bd = base + kSmemB + hp * kBBytes, md = base + kSmemMeta + hp * 1024;
+                const uint32_t bd = base + kSmemB + hp * b_stride, md = base + kSmemMeta + hp * m_stride;
                 tc::mbar_expect_tx(bar(kBarBFull + hp), b_bytes + 8u * (uint32_t)N);
                 tc::tma_load_4d(bd, &cand_map, bar(kBarBFull + hp), 0, 0, uh, 0);
                 tc::tma_load_4d(bd + b_panel, &cand_map, bar(kBarBFull + hp), 64, 0, uh, 0);
                 tc::bulk_load(md, A.cand_scale + (int64_t)uh * N, 4u * (uint32_t)N, bar(kBarBFull + hp));
-                tc::bulk_load(md + 512, A.cand_slot + (int64_t)uh * N, 4u * (uint32_t)N, bar(kBarBFull + hp));
+                tc::bulk_load(md + slot_off, A.cand_slot + (int64_t)uh * N, 4u * (uint32_t)N, bar(kBarBFull + hp));
                 for (int t = 0; ok && t < nt; ++t, ++i) {
                     const int st = i % kStages;
                     ok = tc::mbar_wait(bar(kBarEmpty + st), ((i / kStages) & 1) ^ 1, abort_flag, A.status);
@@ -115,22 +118,28 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             bool ok = true;
             int i = 0, hc = 0;
             for (int uh = blockIdx.x; ok && uh < A.n_heads; uh += gridDim.x, ++hc) {
-                const int hp = hc & 1;
-                ok = tc::mbar_wait(bar(kBarBFull + hp), (hc >> 1) & 1, abort_flag, A.status);
-                const uint32_t bd = base + kSmemB + hp * kBBytes;
+                const int hp = hc % n_bbuf;
+                ok = tc::mbar_wait(bar(kBarBFull + hp), (hc / n_bbuf) & 1, abort_flag, A.status);
+                const uint32_t bd = base + kSmemB + hp * b_stride;
                 for (int t = 0; ok && t < nt; ++t, ++i) {
-                    const int st = i % kStages, set = i % kSets;
-                    ok = tc::mbar_wait(bar(kBarFull + st), (i / kStages) & 1, abort_flag, A.status) &&
-                         tc::mbar_wait(bar(kBarSetFree + set), ((i / kSets) & 1) ^ 1, abort_flag, A.status);
+                    const int st = i % kStages, set = i % n_sets;
+                    // Barriers go by team (tile i belongs to team i mod 4), accumulators by i mod n_sets: the accumulator
+                    // of tile i was last used by tile i - n_sets, whose team signals on its own barrier.  (One barrier per
+                    // accumulator would be waited on by two teams two phases apart, which a parity cannot tell apart.)
+                    ok = tc::mbar_wait(bar(kBarFull + st), (i / kStages) & 1, abort_flag, A.status);
+                    if (ok && i >= n_sets) {
+                        const int j = i - n_sets;
+                        ok = tc::mbar_wait(bar(kBarSetFree + (j & 3)), (j >> 2) & 1, abort_flag, A.status);
+                    }
                     if (!ok) break;
                     tc::tc_fence_after();
                     const uint32_t a = base + st * kStageBytes;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        tc::umma_bf16(tmem + 128 * set, tc::smem_desc_sw128(a + (j >> 2) * kPanel, (j & 3) * 32),
+                        tc::umma_bf16(tmem + set_cols * set, tc::smem_desc_sw128(a + (j >> 2) * kPanel, (j & 3) * 32),
                                       tc::smem_desc_sw128(bd + (j >> 2) * b_panel, (j & 3) * 32), idesc, j > 0);
                     tc::umma_commit(bar(kBarEmpty + st));
-                    tc::umma_commit(bar(kBarAccFull + set));
+                    tc::umma_commit(bar(kBarAccFull + (i & 3)));
                 }
                 if (ok) tc::umma_commit(bar(kBarBEmpty + hp));
             }
@@ -138,13 +147,13 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     } else {
         const int team = (warp - 2) >> 2, wq = warp & 3;
         const int row = 32 * wq + lane;                              // TMEM lane = token of the tile
-        const uint32_t trow = tmem + ((uint32_t)(32 * wq) << 16) + 128 * team;   // team = accumulator set (kTeams == kSets)
+        const uint32_t tlane = tmem + ((uint32_t)(32 * wq) << 16);
         const uint32_t wrow = base + kSmemStash + team * 4096 + row * 32;
         bool ok = true;
         int hc = 0;
         for (int uh = blockIdx.x; uh < A.n_heads; uh += gridDim.x, ++hc) {
-            const int u = uh / A.Hkv, hp = hc & 1;
-            const uint32_t md = base + kSmemMeta + hp * 1024;
+            const int u = uh / A.Hkv, hp = hc % n_bbuf;
+            const uint32_t md = base + kSmemMeta + hp * m_stride;
             const int n_text = A.cand_count[2 * uh], n_vis = A.cand_count[2 * uh + 1];
             const bool intra = A.strategy[u] == 0;
             const int t0 = (n_text + 31) & ~31;
@@ -152,8 +161,9 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             const int nb_all = (end_all + 15) >> 4;                  // blocks of 16 columns that hold candidates
             bool b_ready = false;
             for (int t = 0; t < nt; ++t) {                           // tile number i of this CTA's sequence goes to team i mod 4
-                const int i = hc * nt + t, st = i % kStages;
+                const int i = hc * nt + t, st = i % kStages, set = i % n_sets;
                 if ((i & (kTeams - 1)) != team) continue;
+                const uint32_t trow = tlane + set_cols * set;
                 const int token = t * kTile + row;
                 const bool in_range = token < A.L;
                 const int my_mod = in_range ? A.modality[(int64_t)u * A.L + token] : 0;
@@ -186,10 +196,10 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bar(kBarEmpty + st));
                 if (!b_ready) {                                      // scales and slots of this head have landed
-                    ok = ok && tc::mbar_wait(bar(kBarBFull + hp), (hc >> 1) & 1, abort_flag, A.status);
+                    ok = ok && tc::mbar_wait(bar(kBarBFull + hp), (hc / n_bbuf) & 1, abort_flag, A.status);
                     b_ready = true;
                 }
-                ok = ok && tc::mbar_wait(bar(kBarAccFull + team), (i / kSets) & 1, abort_flag, A.status);
+                ok = ok && tc::mbar_wait(bar(kBarAccFull + team), (i >> 2) & 1, abort_flag, A.status);
                 tc::tc_fence_after();
                 float best = -INFINITY;
                 int best_cc = -1;
@@ -235,7 +245,7 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                         if (w.y == best) idx = 4 * q4 + 1;
                         if (w.x == best) idx = 4 * q4;
                     }
-                    slot = __float_as_int(tc::lds32(md + 512 + (best_cc + idx) * 4));
+                    slot = __float_as_int(tc::lds32(md + slot_off + (best_cc + idx) * 4));
                 }
                 if (in_range && my_rank >= 0 && ok) {                // a non-pivot: report its match
                     float sim = 0.f;
