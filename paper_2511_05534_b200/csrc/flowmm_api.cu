@@ -343,11 +343,16 @@ flowmm_status run_layer_flow(const flowmm_params &p, const float *cross_mass, fl
     return FLOWMM_OK;
 }
 
+// cross_mass != nullptr: the launch also applies Eq. 6 and the theta rule to the final masses (rho may be nullptr)
 flowmm_status run_select(const flowmm_params &p, const float *importance, int32_t *retained, int32_t *evicted,
-                         cudaStream_t st) {
+                         cudaStream_t st, const float *cross_mass = nullptr, float *rho = nullptr,
+                         int32_t *strategy = nullptr) {
     const int threads = p.seq_len <= 2048 ? 256 : p.seq_len <= 8192 ? 512 : kSelectThreads;
+    SelectFlow f;
+    f.cross_mass = cross_mass; f.rho = rho; f.strategy = strategy; f.Hq = p.n_q_heads; f.Hkv = p.n_kv_heads;
+    f.theta = p.theta; f.flow_mode = p.flow_mode;
     select_topb_kernel<<<p.n_units * p.n_kv_heads, threads, 0, st>>>(importance, p.seq_len, p.n_keep, p.window,
-                                                                           p.keep_window, retained, evicted);
+                                                                           p.keep_window, retained, evicted, f);
     FLOWMM_LAUNCHED("select_topb");
     return FLOWMM_OK;
 }
@@ -355,7 +360,8 @@ flowmm_status run_select(const flowmm_params &p, const float *importance, int32_
 
 flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
                            const uint8_t *mod, const int32_t *retained, const int32_t *evicted,
-                           const int32_t *strategy, int32_t *match, float *match_sim, void *ws, cudaStream_t st) {
+                           const int32_t *strategy, int32_t *match, float *match_sim, void *ws, cudaStream_t st,
+                           int2 *tokmap) {
     const int UH = p.n_units * p.n_kv_heads, E = p.seq_len - p.n_keep;
     MatchPrepArgs g;
     g.k = k; g.importance = importance; g.modality = mod;
@@ -386,6 +392,7 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
         mst::Args a;
         a.cand_count = g.cand_count; a.cand_slot = g.cand_slot; a.rank = g.rank; a.strategy = strategy;
         a.cand_scale = g.cand_scale; a.modality = mod; a.match = match; a.match_sim = match_sim;
+        a.tokmap = tokmap; a.merge_mode = p.merge_mode;
         a.status = at<int>(ws, y.status);
         a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.E = E; a.Ctot = y.c_tot; a.n_heads = UH;
         if (cudaFuncSetAttribute(mst::match_small_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -418,12 +425,13 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     return FLOWMM_OK;
 }
 
+// tokmap != nullptr (only with the short-list tensor-core kernel): also write the tensor-core merge's table
 flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
                         const uint8_t *mod, const int32_t *retained, const int32_t *evicted, const int32_t *strategy,
-                        int32_t *match, float *match_sim, void *ws, cudaStream_t st) {
+                        int32_t *match, float *match_sim, void *ws, cudaStream_t st, int2 *tokmap = nullptr) {
     const int E = p.seq_len - p.n_keep;
     if (E == 0) return FLOWMM_OK;
-    if (use_tc(p)) return run_match_tc(p, y, k, importance, mod, retained, evicted, strategy, match, match_sim, ws, st);
+    if (use_tc(p)) return run_match_tc(p, y, k, importance, mod, retained, evicted, strategy, match, match_sim, ws, st, tokmap);
     float *rn = at<float>(ws, y.rn);
     const int64_t rows = (int64_t)p.n_units * p.n_kv_heads * p.seq_len;
     const int lanes = p.head_dim / (p.dtype == FLOWMM_BF16 ? 8 : 4);
@@ -449,9 +457,17 @@ flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, 
     return FLOWMM_OK;
 }
 
+// Few slots per head: Eq. 5 as a product with the slot-by-token weight matrix on the tensor cores.
+// (Below 65536 tokens a slot's fixed-point weight sum cannot overflow.)
+bool merge_is_tc(const flowmm_params &p) {
+    return p.seq_len > p.n_keep && p.dtype == FLOWMM_BF16 && p.head_dim == 128 && p.n_keep <= mtc::kMaxSlots &&
+           p.seq_len < 65536 && p.path != FLOWMM_PATH_SIMT;
+}
+
+// map_ready: the (slot, weight) table of the tensor-core merge has been written already (by the matching kernel)
 flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, const void *v,
                         const int32_t *retained, const int32_t *evicted, const int32_t *match, const float *match_sim,
-                        void *k_out, void *v_out, void *ws, cudaStream_t st) {
+                        void *k_out, void *v_out, void *ws, cudaStream_t st, bool map_ready = false) {
     const int E = p.seq_len - p.n_keep, UH = p.n_units * p.n_kv_heads;
     MergeArgs m;
     m.k = k; m.v = v; m.k_out = k_out; m.v_out = v_out; m.retained = retained;
@@ -463,14 +479,15 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
         m.ks[i] = p.k_stride[i]; m.vs[i] = p.v_stride[i]; m.kos[i] = p.ko_stride[i]; m.vos[i] = p.vo_stride[i];
     }
     // few slots per head: Eq. 5 as a product with the slot-by-token weight matrix on the tensor cores
-    if (E > 0 && p.dtype == FLOWMM_BF16 && p.head_dim == 128 && p.n_keep <= mtc::kMaxSlots && p.seq_len < 65536 &&
-        p.path != FLOWMM_PATH_SIMT) {       // (below 65536 tokens a slot's fixed-point weight sum cannot overflow)
+    if (merge_is_tc(p)) {
         mtc::MapArgs ma;
         ma.retained = retained; ma.evicted = evicted; ma.match = match; ma.match_sim = match_sim;
         ma.tokmap = at<int2>(ws, y.tokmap); ma.L = p.seq_len; ma.B = p.n_keep; ma.E = E; ma.merge_mode = p.merge_mode;
         const int longest = E > p.n_keep ? E : p.n_keep;
-        mtc::merge_map_kernel<<<dim3((longest + 255) / 256, UH), 256, 0, st>>>(ma);
-        FLOWMM_LAUNCHED("merge_map");
+        if (!map_ready) {
+            mtc::merge_map_kernel<<<dim3((longest + 255) / 256, UH), 256, 0, st>>>(ma);
+            FLOWMM_LAUNCHED("merge_map");
+        }
         CUtensorMap kmap, vmap;
         const uint64_t dims[4] = {128, (uint64_t)p.seq_len, (uint64_t)p.n_kv_heads, (uint64_t)p.n_units};
         const uint64_t ksb[3] = {(uint64_t)p.k_stride[2] * 2, (uint64_t)p.k_stride[1] * 2, (uint64_t)p.k_stride[0] * 2};
@@ -630,16 +647,21 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
     float *cross_mass = at<float>(ws, y.cross_mass);
     int n_parts = 0;
     FLOWMM_TRY(run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, st, &n_parts));
+    bool flow_in_select = false;
     if (n_parts == 0) {
-        FLOWMM_TRY(run_layer_flow(*p, cross_mass, rho, strategy, st));
+        flow_in_select = true;               // the masses are final: Eq. 6 and the theta rule ride along with the selection
     } else {
         flow_from_parts_kernel<<<p->n_units, 256, 0, st>>>(at<float>(ws, y.cross_part), n_parts, p->n_q_heads, p->window,
                                                            p->theta, p->flow_mode, cross_mass, rho, strategy);
         FLOWMM_LAUNCHED("flow_from_parts");
     }
-    FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st));
-    FLOWMM_TRY(run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws, st));
-    FLOWMM_TRY(run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws, st));
+    if (flow_in_select) FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st, cross_mass, rho, strategy));
+    else FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st));
+    // when both the short-list matching kernel and the tensor-core merge apply, the former writes the latter's table
+    const bool map_in_match = p->seq_len > p->n_keep && use_tc(*p) && y.c_tot <= mst::kMaxCols && merge_is_tc(*p);
+    FLOWMM_TRY(run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws, st,
+                         map_in_match ? at<int2>(ws, y.tokmap) : nullptr));
+    FLOWMM_TRY(run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws, st, map_in_match));
     return FLOWMM_OK;
 }
 

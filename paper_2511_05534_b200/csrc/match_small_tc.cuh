@@ -42,8 +42,9 @@ struct Args {
     const uint8_t *modality;
     int *match;
     float *match_sim;
+    int2 *tokmap;          // nullptr, or [UH, L]: the (slot, weight) table of the tensor-core merge, written here instead of by merge_map_kernel
     int *status;
-    int Hkv, L, E, Ctot, n_heads;
+    int Hkv, L, E, Ctot, n_heads, merge_mode;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -252,6 +253,10 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                     if (slot >= 0 && ssq > 0.f) sim = best * rsqrtf(ssq);
                     A.match[(int64_t)uh * A.E + my_rank] = slot;
                     A.match_sim[(int64_t)uh * A.E + my_rank] = sim;
+                    if (A.tokmap)                                    // same entry as merge_map_kernel would write
+                        A.tokmap[(int64_t)uh * A.L + token] = make_int2(slot, __float_as_int(A.merge_mode == 1 ? 1.f : __expf(sim - 1.f)));
+                } else if (in_range && ok && A.tokmap) {             // a pivot: its own slot with weight 1
+                    A.tokmap[(int64_t)uh * A.L + token] = make_int2((-my_rank - 2) | (1 << 30), __float_as_int(1.f));
                 }
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bar(kBarBEmpty + hp));      // done with this head's scales and slots for this tile

@@ -29,7 +29,7 @@ struct MatchPrepArgs {
     float *cand_scale;           // [UH, Ctot]
     int *cand_slot;              // [UH, Ctot]
     int *cand_count;             // [UH, 2]  admissible text / visual pivots
-    int *rank;                   // [UH, L]  position in the non-pivot list, or -1 for a pivot
+    int *rank;                   // [UH, L]  position in the non-pivot list, or -(s + 2) for the pivot of slot s
     uint8_t *tile_mod;           // [U, n_rt] per tile of 256 tokens; bit 0: holds text tokens, bit 1: visual tokens
     int Hkv, L, B, E, Ctot, n_rt;
     int copy_here;               // 1: this kernel also gathers the candidate rows; 0: match_gather_kernel does
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(256) match_prepare_kernel(const MatchPrepArgs 
     float *scale_out = A.cand_scale + (int64_t)uh * A.Ctot;
 
     for (int i = tid; i < A.Ctot; i += blockDim.x) { slot_out[i] = -1; scale_out[i] = __int_as_float(0x7FC00000); }   // NaN: no candidate here
-    for (int s = tid; s < A.B; s += blockDim.x) rank[ret[s]] = -1;
+    for (int s = tid; s < A.B; s += blockDim.x) rank[ret[s]] = -(s + 2);
     for (int j = tid; j < A.E; j += blockDim.x) rank[evi[j]] = j;
     if (h == 0) {
         for (int t = tid; t < A.n_rt; t += blockDim.x) {

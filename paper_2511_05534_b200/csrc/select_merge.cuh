@@ -17,8 +17,20 @@ __device__ __forceinline__ uint32_t select_key(float v, bool forced) {
 // Section 3.3.1 pivot selection: a radix select finds the B-th largest key, then one ordered
 // sweep writes the pivot positions and the non-pivot positions, both ascending.  Ties at the
 // threshold go to the lower positions.  grid = U*Hkv, block = any multiple of 32 up to 1024.
+// Eq. 6 and the theta rule riding along with the selection (cross_mass == nullptr: not asked for): the block of a
+// unit's first KV head applies them, one thread, same arithmetic as layer_flow_kernel.
+struct SelectFlow {
+    const float *cross_mass;     // [U, Hq] final per-head masses
+    float *rho;                  // [U] or nullptr
+    int *strategy;               // [U]
+    int Hq, Hkv;
+    float theta;
+    int flow_mode;
+};
+
 __global__ void __launch_bounds__(kSelectThreads)
-select_topb_kernel(const float *importance, int L, int B, int W, int keep_window, int *retained, int *evicted) {
+select_topb_kernel(const float *importance, int L, int B, int W, int keep_window, int *retained, int *evicted,
+                   const SelectFlow F) {
     __shared__ int hist[256];
     __shared__ int scratch[33];
     __shared__ uint32_t s_prefix;
@@ -28,6 +40,14 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
     int *ret = retained + (int64_t)blockIdx.x * B;
     int *evi = evicted + (int64_t)blockIdx.x * (L - B);
     const int first_forced = keep_window ? L - W : L;
+    if (F.cross_mass && blockIdx.x % F.Hkv == 0 && tid == nthreads - 1) {
+        const int u = blockIdx.x / F.Hkv;
+        float s = 0.f;
+        for (int g = 0; g < F.Hq; ++g) s += F.cross_mass[(int64_t)u * F.Hq + g] / (float)W;   // a head's total mass is W
+        const float r = s / (float)F.Hq;
+        if (F.rho) F.rho[u] = r;
+        F.strategy[u] = F.flow_mode == 1 ? 0 : F.flow_mode == 2 ? 1 : ((r > F.theta) != (F.flow_mode == 3) ? 1 : 0);
+    }
 
     // radix select, most significant byte first: after the loop `prefix` is the B-th largest key
     uint32_t prefix = 0, mask = 0;
