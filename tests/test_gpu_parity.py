@@ -77,6 +77,29 @@ def test_ragged_shapes(dtype, D):
         _random_case(rng, U, Hq, Hkv, D, L, W, B, dtype, tau=3.0, tau_mode=O.TAU_REL, theta=0.5)
 
 
+def test_short_context_kernel_boundaries():
+    """Shapes around the switch points of the one-pass scoring kernel (32 proxy rows per KV head, up to 8 key
+    tiles), the short-list matching kernel (up to 256 candidate columns, i.e. B <= 224) and the tensor-core merge
+    (B <= 240), with ragged lengths and windows that straddle a tile edge."""
+    rng = np.random.default_rng(23)
+    for (U, Hq, Hkv, L, W, B) in [
+        (2, 2, 2, 333, 32, 40),      # G W = 32, three key tiles, ragged tail
+        (1, 4, 2, 1000, 16, 96),     # G = 2, W = 16, eight key tiles; 96 pivots: 128 candidate columns
+        (2, 1, 1, 129, 32, 1),       # window across the tile edge, a single pivot
+        (1, 2, 2, 1024, 32, 224),    # the longest context of the one-pass kernel; 256 candidate columns
+        (1, 2, 2, 1025, 32, 225),    # one token and one pivot more: two-pass scoring, general matching kernel
+        (1, 2, 1, 600, 32, 240),     # the largest budget of the tensor-core merge
+        (1, 2, 1, 600, 32, 241),     # one more: gather merge
+        (3, 2, 2, 64, 32, 33),       # half of the prompt is the window
+    ]:
+        _random_case(rng, U, Hq, Hkv, 128, L, W, B, F.BF16, tau=3.0, tau_mode=O.TAU_REL, theta=0.5)
+    # every layer forced either way, and pivots all protected (nothing is merged: the compaction alone)
+    _random_case(rng, 2, 2, 2, 128, 640, 32, 64, F.BF16, flow_mode=O.FLOW_FORCE_INTRA, vis_frac=0.8)
+    _random_case(rng, 2, 2, 2, 128, 640, 32, 64, F.BF16, flow_mode=O.FLOW_FORCE_CROSS, merge_mode=O.MERGE_MEAN)
+    _random_case(rng, 1, 2, 2, 128, 640, 32, 64, F.BF16, tau=0.0)
+    _random_case(rng, 1, 2, 2, 128, 300, 32, 100, F.BF16, keep_window=1, tau=float("inf"))
+
+
 def test_degenerate_cases():
     rng = np.random.default_rng(7)
     _random_case(rng, 1, 2, 2, 64, 50, 50, 1, F.F32)                       # one pivot, window = whole prompt
