@@ -195,6 +195,25 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
                                     void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The step before the compression path: the cross-modal interaction ratio of Eq. 6 and Eq. 7 taken
+ * literally, over every query row of the prefill (both the text-to-visual and the visual-to-text
+ * term), instead of over the proxy window that flowmm_score uses.  Causal softmax attention of all
+ * L queries; per query head the attention mass that lands on keys of the other modality than the
+ * query's, summed over the rows; rho = mean over heads of that mass / L; strategy by theta.
+ *   q_full [U, Hq, L, D] with the element strides q_full_stride (unit, head, token); head_dim contiguous
+ *   k      [U, Hkv, L, D] with p->k_stride
+ *   cross_mass [U, Hq] f32 out;  rho [U] f32 out (may be NULL);  strategy [U] int32 out
+ * Of p, the fields n_units, n_q_heads, n_kv_heads, head_dim, seq_len, dtype, softmax_scale, theta,
+ * flow_mode, k_stride and path are used (window, n_keep, tau, q_stride are not).  The work is the
+ * scoring step applied to query tiles of 128 rows, each against the keys up to its last row, so it
+ * costs O(L^2 D) per head.  Scratch: flowmm_full_flow_workspace_bytes; its first word is the device status.
+ */
+flowmm_status flowmm_full_flow_workspace_bytes(const flowmm_params *p, size_t *bytes);
+flowmm_status flowmm_full_flow(const flowmm_params *p, const void *q_full, const int64_t q_full_stride[3],
+                               const void *k, const uint8_t *modality, float *cross_mass, float *rho,
+                               int32_t *strategy, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * The step after the compression path: decode-time attention of one new query per query head over a
  * cache of n_keys rows, Eq. 4 - o = softmax(q . K^T * scale) V - for the full cache or for the
  * compressed one that flowmm_compress_layer wrote.  Every cache row is read once for all G query

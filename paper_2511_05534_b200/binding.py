@@ -30,6 +30,7 @@ EXPORTS = (
     "flowmm_compress_layer", "flowmm_last_device_status", "flowmm_last_launch_count", "flowmm_status_string",
     "flowmm_profile_enable", "flowmm_profile_read", "flowmm_merge_static", "flowmm_selftest_wait_timeout",
     "flowmm_decode_workspace_bytes", "flowmm_decode_attention",
+    "flowmm_full_flow_workspace_bytes", "flowmm_full_flow",
 )
 
 
@@ -123,6 +124,8 @@ def load() -> ctypes.CDLL:
         lib.flowmm_selftest_wait_timeout.restype = ctypes.c_int
         lib.flowmm_decode_workspace_bytes.restype = ctypes.c_int
         lib.flowmm_decode_attention.restype = ctypes.c_int
+        lib.flowmm_full_flow_workspace_bytes.restype = ctypes.c_int
+        lib.flowmm_full_flow.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -170,6 +173,23 @@ def flowmm_score(p: Params, q_win, k, modality, importance, cross_mass, ws):
     cp = p.c(q=q_win, k=k)
     _check(load().flowmm_score(ctypes.byref(cp), _p(q_win), _p(k), _p(modality), _p(importance), _p(cross_mass),
                                _p(ws), ctypes.c_size_t(ws.numel()), _stream()), "flowmm_score")
+
+
+def flowmm_full_flow_workspace_bytes(p: Params) -> int:
+    n = ctypes.c_size_t(0)
+    cp = p.c()
+    _check(load().flowmm_full_flow_workspace_bytes(ctypes.byref(cp), ctypes.byref(n)), "flowmm_full_flow_workspace_bytes")
+    return int(n.value)
+
+
+def flowmm_full_flow(p: Params, q_full, k, modality, cross_mass, rho, strategy, ws):
+    """Eq. 6 and Eq. 7 over every query row of the prefill: q_full [units, q_heads, seq_len, head_dim]."""
+    if q_full.dim() != 4 or q_full.stride(3) != 1:
+        raise ValueError("expected a [units, heads, tokens, head_dim] tensor with contiguous head_dim")
+    cp = p.c(k=k)
+    qs = (ctypes.c_int64 * 3)(q_full.stride(0), q_full.stride(1), q_full.stride(2))
+    _check(load().flowmm_full_flow(ctypes.byref(cp), _p(q_full), qs, _p(k), _p(modality), _p(cross_mass), _p(rho),
+                                   _p(strategy), _p(ws), ctypes.c_size_t(ws.numel()), _stream()), "flowmm_full_flow")
 
 
 def flowmm_layer_flow(p: Params, cross_mass, rho, strategy):

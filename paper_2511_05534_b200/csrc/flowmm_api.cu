@@ -720,6 +720,101 @@ const char *flowmm_status_string(flowmm_status s) {
 
 }  // extern "C"
 
+// ---- full-prefill information flow ---------------------------------------------------------------
+namespace {
+
+constexpr int kFlowTile = 128;      // query rows per scoring call
+
+// Query tile t of n: rows [lo, hi); the first tile takes the remainder so that all others are full.
+void flow_tile(int L, int t, int &lo, int &hi) {
+    const int rem = L % kFlowTile, n_full = L / kFlowTile;
+    if (rem == 0) { lo = t * kFlowTile; hi = lo + kFlowTile; return; }
+    if (t == 0) { lo = 0; hi = rem; return; }
+    lo = rem + (t - 1) * kFlowTile; hi = lo + kFlowTile;
+    (void)n_full;
+}
+int flow_tiles(int L) { return (L + kFlowTile - 1) / kFlowTile; }
+
+// The scoring step's parameters for one query tile: the prompt cut after the tile's last row, the tile as window.
+flowmm_params flow_tile_params(const flowmm_params &p, const int64_t qs[3], int lo, int hi) {
+    flowmm_params t = p;
+    t.seq_len = hi; t.window = hi - lo; t.n_keep = 1; t.keep_window = 0; t.tau = 0.f; t.tau_mode = FLOWMM_TAU_ABS;
+    for (int i = 0; i < 3; ++i) t.q_stride[i] = qs[i];
+    return t;
+}
+
+struct FlowLayout { size_t std_bytes, mod, imp, parts, total; };
+
+FlowLayout flow_layout(const flowmm_params &p, const int64_t qs[3]) {
+    FlowLayout f = {};
+    const int n = flow_tiles(p.seq_len);
+    for (int t = 0; t < n; ++t) {
+        int lo, hi;
+        flow_tile(p.seq_len, t, lo, hi);
+        const size_t need = make_layout(flow_tile_params(p, qs, lo, hi)).total;
+        if (need > f.std_bytes) f.std_bytes = need;
+    }
+    size_t o = align256(f.std_bytes);
+    f.mod = o; o += align256((size_t)p.n_units * p.seq_len);
+    f.imp = o; o += align256((size_t)p.n_units * p.n_kv_heads * p.seq_len * 4);
+    f.parts = o; o += align256((size_t)n * p.n_units * p.n_q_heads * 4);
+    f.total = o;
+    return f;
+}
+
+flowmm_status validate_flow(const flowmm_params *p) {
+    if (!p) return FLOWMM_ERR_NULL;
+    flowmm_params t = *p;
+    t.window = 1; t.n_keep = 1; t.keep_window = 0; t.tau = 0.f; t.tau_mode = FLOWMM_TAU_ABS;   // not used here
+    return validate(&t);
+}
+
+}  // namespace
+
+extern "C" flowmm_status flowmm_full_flow_workspace_bytes(const flowmm_params *p, size_t *bytes) {
+    if (!bytes) return FLOWMM_ERR_NULL;
+    FLOWMM_TRY(validate_flow(p));
+    const int64_t dense[3] = {(int64_t)p->n_q_heads * p->seq_len * p->head_dim, (int64_t)p->seq_len * p->head_dim, p->head_dim};
+    *bytes = flow_layout(*p, dense).total;
+    return FLOWMM_OK;
+}
+
+extern "C" flowmm_status flowmm_full_flow(const flowmm_params *p, const void *q_full, const int64_t q_full_stride[3],
+                                          const void *k, const uint8_t *modality, float *cross_mass, float *rho,
+                                          int32_t *strategy, void *ws, size_t ws_bytes, void *cuda_stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    profile_begin(st);
+    FLOWMM_TRY(validate_flow(p));
+    if (!q_full || !q_full_stride || !k || !modality || !cross_mass || !strategy || !ws) return FLOWMM_ERR_NULL;
+    if (!aligned16(q_full) || !aligned16(k) || !strides_ok(q_full_stride, p->head_dim) || !strides_ok(p->k_stride, p->head_dim) ||
+        (reinterpret_cast<uintptr_t>(ws) & 255))
+        return FLOWMM_ERR_ALIGN;
+    const FlowLayout f = flow_layout(*p, q_full_stride);
+    if (ws_bytes < f.total) return FLOWMM_ERR_WORKSPACE;
+    FLOWMM_TRY(check_device());
+    if (cudaMemsetAsync(ws, 0, 4, st) != cudaSuccess) return FLOWMM_ERR_CUDA;       // the status word
+    const int n_tiles = flow_tiles(p->seq_len), n = p->n_units * p->n_q_heads;
+    const size_t esize = p->dtype == FLOWMM_BF16 ? 2 : 4;
+    uint8_t *mod = at<uint8_t>(ws, f.mod);
+    float *imp = at<float>(ws, f.imp), *parts = at<float>(ws, f.parts);
+    for (int t = 0; t < n_tiles; ++t) {
+        int lo, hi;
+        flow_tile(p->seq_len, t, lo, hi);
+        const flowmm_params tp = flow_tile_params(*p, q_full_stride, lo, hi);
+        const Layout y = make_layout(tp);
+        // the scoring kernels index the modality map with the cut prompt's length as the row pitch
+        if (cudaMemcpy2DAsync(mod, (size_t)hi, modality, (size_t)p->seq_len, (size_t)hi, (size_t)p->n_units,
+                              cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return FLOWMM_ERR_CUDA;
+        const char *q_tile = static_cast<const char *>(q_full) + (size_t)lo * (size_t)q_full_stride[2] * esize;
+        FLOWMM_TRY(run_score(tp, y, q_tile, k, mod, imp, parts + (size_t)t * n, ws, st));
+    }
+    full_flow_reduce_kernel<<<p->n_units, 64, 0, st>>>(parts, n_tiles, n, p->n_q_heads, p->seq_len, p->theta, p->flow_mode,
+                                                       cross_mass, rho, strategy);
+    FLOWMM_LAUNCHED("full_flow_reduce");
+    return FLOWMM_OK;
+}
+
 // ---- decode-step attention over a cache ---------------------------------------------------------
 namespace {
 

@@ -286,6 +286,26 @@ __global__ void flow_from_parts_kernel(const float *cross_part, int n_chunk, int
     }
 }
 
+// Full-prefill flow: per-head masses of the query tiles added up in tile order, then Eq. 6 over all L rows
+// and the theta rule.  parts [n_tiles][U * Hq]; one block per unit, one thread per query head.
+__global__ void full_flow_reduce_kernel(const float *parts, int n_tiles, int n, int Hq, int L, float theta, int flow_mode,
+                                        float *cross_mass, float *rho, int *strategy) {
+    const int u = blockIdx.x;
+    for (int g = threadIdx.x; g < Hq; g += blockDim.x) {
+        float s = 0.f;
+        for (int t = 0; t < n_tiles; ++t) s += parts[(int64_t)t * n + (int64_t)u * Hq + g];
+        cross_mass[(int64_t)u * Hq + g] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int g = 0; g < Hq; ++g) s += cross_mass[(int64_t)u * Hq + g] / (float)L;   // a head's total mass is L
+        const float r = s / (float)Hq;
+        if (rho) rho[u] = r;
+        strategy[u] = flow_mode == 1 ? 0 : flow_mode == 2 ? 1 : ((r > theta) != (flow_mode == 3) ? 1 : 0);
+    }
+}
+
 // Reciprocal Euclidean norm of every key row (0 for a zero row).  One group of D/kVec lanes per row.
 template <typename T>
 __global__ void inv_norm_kernel(const void *k_, int64_t n_rows, int Hkv, int L, int D, int64_t s0, int64_t s1,

@@ -93,6 +93,33 @@ def test_score_equals_library_softmax(G):
     np.testing.assert_allclose(imp[0], exp_imp, rtol=1e-11, atol=1e-15)
 
 
+def test_whole_prompt_as_window_is_the_full_prefill_flow():
+    """With the window equal to the prompt every query row is a proxy row, and the masses of Eq. 7 are the literal
+    sums over all (query, key) pairs, text-to-visual and visual-to-text: checked against scipy's causal softmax,
+    against the uniform-attention closed form, and against the two one-modality cases."""
+    rng = np.random.default_rng(29)
+    L, D = 37, 16
+    p = params(Hq=2, Hkv=1, D=D, L=L, W=L, B=1)
+    q, k, v, m = rand_unit(rng, p, vis_frac=0.5)
+    _, cross, total = O.score(p, q, k, m)
+    mask = np.where(np.arange(L)[None, :] <= np.arange(L)[:, None], 0.0, -np.inf)
+    other = m[0][None, :] != m[0][:, None]
+    for g in range(2):
+        a = softmax(q[0, g].astype(np.float64) @ k[0, 0].astype(np.float64).T / math.sqrt(D) + mask, axis=-1)
+        v2t = a[(m[0] == 1)[:, None] & (m[0] == 0)[None, :]].sum()       # visual queries on text keys
+        t2v = a[(m[0] == 0)[:, None] & (m[0] == 1)[None, :]].sum()
+        assert abs(cross[0, g] - (v2t + t2v)) < 1e-12 and abs(cross[0, g] - a[other].sum()) < 1e-12
+        assert abs(total[0, g] - L) < 1e-12
+    q[:] = 0                                                             # uniform rows: alpha[j, i] = 1 / (j + 1)
+    _, cross, _ = O.score(p, q, k, m)
+    exp = sum(Fraction(sum(1 for i in range(j + 1) if m[0, i] != m[0, j]), j + 1) for j in range(L))
+    np.testing.assert_allclose(cross[0], float(exp), rtol=1e-13)
+    for vis in (0, 1):
+        _, cross, total = O.score(p, rng.standard_normal(q.shape).astype(np.float32), k, np.full_like(m, vis))
+        rho, strat = O.layer_flow(p, cross, total)
+        assert np.all(cross == 0) and rho[0] == 0 and strat[0] == O.INTRA
+
+
 def test_score_invariants():
     rng = np.random.default_rng(2)
     for (Hq, Hkv, D, L, W) in [(4, 2, 8, 37, 5), (3, 3, 16, 64, 64), (8, 1, 4, 19, 1)]:
