@@ -60,6 +60,7 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // Where everything lives inside the caller's workspace.  One layout serves every entry point.
 struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
+    size_t row_cross;          // flow-only statistics pass: the other-modality part of every partial row sum
     size_t row_part, cross_part, rn, sort_a, sort_b, mem_tok, mem_w, piece_desc, off, piece_off, part_off, partial, ticket, slot_done;
     size_t cand_k, cand_scale, cand_slot, cand_count, rank, tile_mod, negc;
     size_t tokmap;             // [UH, L] (slot, weight) of every token position, for the tensor-core merge
@@ -141,6 +142,7 @@ Layout make_layout(const flowmm_params &p) {
     const size_t max_chunk1 = (size_t)(y.n_chunk1 > 4 * y.tc_n_chunk ? y.n_chunk1 : 4 * y.tc_n_chunk);
     const size_t max_chunk2 = (size_t)(y.n_chunk2 > 8 * y.n_rt ? y.n_chunk2 : 8 * y.n_rt);
     y.row_part = take(U * Hq * W * max_chunk1 * 8);
+    y.row_cross = take(U * Hq * W * max_chunk1 * 4);
     y.cross_part = take(U * Hq * max_chunk2 * 4);
     y.negc = take(U * Hkv * (size_t)y.gw_pad * 4);
     y.rn = take(U * Hkv * L * 4);
@@ -743,7 +745,41 @@ flowmm_params flow_tile_params(const flowmm_params &p, const int64_t qs[3], int 
     return t;
 }
 
-struct FlowLayout { size_t std_bytes, mod, imp, parts, total; };
+struct FlowLayout { size_t std_bytes, mod, imp, parts, bits, total; };
+
+// One query tile of the full-prefill flow on the tensor cores: the statistics pass alone, with the row sums split by
+// key modality, then the per-head join.  `tp` is the tile's scoring problem (prompt cut after the tile, tile = window).
+flowmm_status run_flow_tile_tc(const flowmm_params &tp, const Layout &y, const void *q_tile, const void *k,
+                               const uint8_t *modality, int mod_pitch, const uint32_t *modbits, int mod_words,
+                               float *cross_out, void *ws, cudaStream_t st) {
+    const int UH = tp.n_units * tp.n_kv_heads, G = tp.n_q_heads / tp.n_kv_heads, W = tp.window;
+    ScoreTcArgs a = {};
+    a.row_part = at<float2>(ws, y.row_part); a.row_cross = at<float>(ws, y.row_cross); a.modality = modality;
+    a.modbits = modbits; a.mod_words = mod_words; a.mod_pitch = mod_pitch; a.status = at<int>(ws, y.status);
+    a.Hq = tp.n_q_heads; a.Hkv = tp.n_kv_heads; a.G = G; a.W = W; a.L = tp.seq_len; a.GW = G * W; a.GWpad = y.gw_pad;
+    a.n_qt = y.tc_n_qt; a.n_chunk = y.tc_n_chunk; a.tiles_per_chunk = y.tc_tiles_per_chunk; a.n_rt = y.n_rt;
+    a.a_heads = G < tcs::kRows / W ? G : tcs::kRows / W;
+    a.n_items1 = UH * a.n_qt * a.n_chunk;
+    const float scale = tp.softmax_scale != 0.f ? tp.softmax_scale : 1.f / sqrtf((float)tp.head_dim);
+    a.scale_log2 = scale * kLog2e;
+    CUtensorMap qa, k256;
+    const uint64_t qd[4] = {128, (uint64_t)W, (uint64_t)tp.n_q_heads, (uint64_t)tp.n_units};
+    const uint64_t qs[3] = {(uint64_t)tp.q_stride[2] * 2, (uint64_t)tp.q_stride[1] * 2, (uint64_t)tp.q_stride[0] * 2};
+    const uint64_t kd[4] = {128, (uint64_t)tp.seq_len, (uint64_t)tp.n_kv_heads, (uint64_t)tp.n_units};
+    const uint64_t ks[3] = {(uint64_t)tp.k_stride[2] * 2, (uint64_t)tp.k_stride[1] * 2, (uint64_t)tp.k_stride[0] * 2};
+    const uint32_t bqa[4] = {64, (uint32_t)W, (uint32_t)a.a_heads, 1}, bk256[4] = {64, tcs::Big::kCols, 1, 1};
+    if (!tc::make_bf16_map(&qa, q_tile, 4, qd, qs, bqa) || !tc::make_bf16_map(&k256, k, 4, kd, ks, bk256)) return FLOWMM_ERR_CUDA;
+    if (cudaFuncSetAttribute(score_stats_tc_kernel<tcs::Big, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tcs::Big::kSmemBytes) != cudaSuccess)
+        return FLOWMM_ERR_CUDA;
+    const int sms = tc::sm_count();
+    score_stats_tc_kernel<tcs::Big, true><<<a.n_items1 < sms ? a.n_items1 : sms, tcs::kThreads, tcs::Big::kSmemBytes, st>>>(qa, k256, a);
+    FLOWMM_LAUNCHED("flow_stats_tc");
+    const int n_heads = tp.n_units * tp.n_q_heads;
+    flow_combine_kernel<<<(n_heads + 7) / 8, 256, 0, st>>>(a.row_part, a.row_cross, 4 * a.n_chunk, G, W, tp.n_kv_heads, n_heads, cross_out);
+    FLOWMM_LAUNCHED("flow_combine");
+    return FLOWMM_OK;
+}
 
 FlowLayout flow_layout(const flowmm_params &p, const int64_t qs[3]) {
     FlowLayout f = {};
@@ -758,6 +794,7 @@ FlowLayout flow_layout(const flowmm_params &p, const int64_t qs[3]) {
     f.mod = o; o += align256((size_t)p.n_units * p.seq_len);
     f.imp = o; o += align256((size_t)p.n_units * p.n_kv_heads * p.seq_len * 4);
     f.parts = o; o += align256((size_t)n * p.n_units * p.n_q_heads * 4);
+    f.bits = o; o += align256((size_t)p.n_units * ((p.seq_len + 31) / 32 + 8) * 4);
     f.total = o;
     return f;
 }
@@ -797,11 +834,22 @@ extern "C" flowmm_status flowmm_full_flow(const flowmm_params *p, const void *q_
     const size_t esize = p->dtype == FLOWMM_BF16 ? 2 : 4;
     uint8_t *mod = at<uint8_t>(ws, f.mod);
     float *imp = at<float>(ws, f.imp), *parts = at<float>(ws, f.parts);
+    uint32_t *bits = at<uint32_t>(ws, f.bits);
+    const int mod_words = (p->seq_len + 31) / 32 + 8;                  // + slack: whole 256-key tiles are indexed
+    if (use_tc(*p)) {
+        pack_modality_kernel<<<dim3((mod_words + 7) / 8, p->n_units), 256, 0, st>>>(modality, p->seq_len, mod_words, bits);
+        FLOWMM_LAUNCHED("pack_modality");
+    }
     for (int t = 0; t < n_tiles; ++t) {
         int lo, hi;
         flow_tile(p->seq_len, t, lo, hi);
         const flowmm_params tp = flow_tile_params(*p, q_full_stride, lo, hi);
         const Layout y = make_layout(tp);
+        const char *q_tile_tc = static_cast<const char *>(q_full) + (size_t)lo * (size_t)q_full_stride[2] * esize;
+        if (use_tc_score(tp)) {            // full tiles on the tensor cores: one pass, no importance
+            FLOWMM_TRY(run_flow_tile_tc(tp, y, q_tile_tc, k, modality, p->seq_len, bits, mod_words, parts + (size_t)t * n, ws, st));
+            continue;
+        }
         // the scoring kernels index the modality map with the cut prompt's length as the row pitch
         if (cudaMemcpy2DAsync(mod, (size_t)hi, modality, (size_t)p->seq_len, (size_t)hi, (size_t)p->n_units,
                               cudaMemcpyDeviceToDevice, st) != cudaSuccess)

@@ -32,6 +32,10 @@ struct ScoreTcArgs {
     int a_heads, b_heads;        // query heads one A box (pass 1) / B box (pass 2) delivers
     int n_items1, n_items2;
     float scale_log2;
+    // flow-only variant of pass 1 (full-prefill flow): the row sums also split off the keys of the other modality
+    float *row_cross;            // [UH*GW, 4*n_chunk] that part of the sum, same scaling as row_part
+    const uint32_t *modbits;     // [U, mod_words] key modality, 32 keys per word (bit j of word w: key 32 w + j is visual)
+    int mod_words, mod_pitch;    // words per unit in modbits; row pitch of `modality` (the uncut prompt's length)
 };
 
 // max of 32 values with three-input maxima
@@ -47,7 +51,9 @@ __device__ __forceinline__ float max32(const float (&v)[32]) {
 
 // ---------------------------------------------------------------------------------------------
 // Pass 1.  item = (unit*head, tile of 256 proxy rows, key chunk).
-template <class S>
+// kFlow: also keep, per row, the part of the exp-sum that falls on keys of the other modality than the row's token
+// (a chunk of 32 keys is usually of one modality: then it costs one comparison; only mixed chunks go element by element).
+template <class S, bool kFlow = false>
 __global__ void __launch_bounds__(tcs::kThreads, 1)
 score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                       const ScoreTcArgs A) {
@@ -85,6 +91,18 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
             if (p.empty()) continue;
             const int kc = item % A.n_chunk, qt = (item / A.n_chunk) % A.n_qt, uh = item / (A.n_chunk * A.n_qt);
             float m[2] = {kNegBig, kNegBig}, l[2] = {0.f, 0.f};
+            float lc[2] = {0.f, 0.f};
+            bool my_vis[2] = {false, false};
+            const uint32_t *bits = nullptr;
+            if constexpr (kFlow) {
+                const int u = uh / A.Hkv;
+                bits = A.modbits + (int64_t)u * A.mod_words;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int pa = A.L - A.W + ((qt * tcs::kItemRows + h * tcs::kRows + row_in_half) % A.W);
+                    my_vis[h] = A.modality[(int64_t)u * A.mod_pitch + pa] != 0;
+                }
+            }
             for (int t = 0; ok && t < p.n_tiles; ++t) {
                 const int kb = p.b1 + t * S::kCols;
                 const int ncols = min(S::kCols, p.cols_total - t * S::kCols);
@@ -100,6 +118,9 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
                             const int k0 = kb + ch * 32;
                             float mx;
                             float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
+                            float addc = 0.f;                            // kFlow: the other-modality part of this chunk's sum
+                            uint32_t other = 0;
+                            if constexpr (kFlow) other = my_vis[h] ? ~bits[k0 >> 5] : bits[k0 >> 5];
                             if (k0 + 32 <= A.L - A.W + 1) {              // no key of this chunk is masked for any row
                                 float raw[32];
 #pragma unroll
@@ -115,6 +136,14 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
                                     a23 = tc::fadd2(a23, make_float2(tc::ex2(x23.x), tc::ex2_fma(x23.y)));   // every fourth one on the FMA pipe
                                 }
                                 add0 = a01.x; add1 = a01.y; add2 = a23.x; add3 = a23.y;
+                                if constexpr (kFlow) {
+                                    if (other == 0xFFFFFFFFu) addc = (add0 + add1) + (add2 + add3);
+                                    else if (other != 0u) {
+#pragma unroll
+                                        for (int j = 0; j < 32; ++j)
+                                            addc += ((other >> j) & 1u) ? tc::ex2(fmaf(raw[j], A.scale_log2, -mx)) : 0.f;
+                                    }
+                                }
                             } else {
                                 float s[32];
 #pragma unroll
@@ -128,10 +157,16 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
                                     add2 += tc::ex2(s[j + 2] - mx);
                                     add3 += tc::ex2(s[j + 3] - mx);
                                 }
+                                if constexpr (kFlow) {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) addc += ((other >> j) & 1u) ? tc::ex2(s[j] - mx) : 0.f;
+                                }
                             }
                             float add = (add0 + add1) + (add2 + add3);
-                            if (mx < 0.5f * kNegBig) add = 0.f;          // nothing visible yet: exp2(0) terms are not real
-                            l[h] = l[h] * tc::ex2(m[h] - mx) + add;
+                            if (mx < 0.5f * kNegBig) { add = 0.f; addc = 0.f; }   // nothing visible yet: exp2(0) terms are not real
+                            const float carry = tc::ex2(m[h] - mx);
+                            l[h] = l[h] * carry + add;
+                            if constexpr (kFlow) lc[h] = lc[h] * carry + addc;
                             m[h] = mx;
                         });
                     }
@@ -142,12 +177,47 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int r = qt * tcs::kItemRows + h * tcs::kRows + row_in_half;
-                if (h < p.n_halves && r < A.GW)
+                if (h < p.n_halves && r < A.GW) {
                     A.row_part[((int64_t)uh * A.GW + r) * (4 * A.n_chunk) + 4 * kc + colq] = make_float2(m[h], l[h]);
+                    if constexpr (kFlow) A.row_cross[((int64_t)uh * A.GW + r) * (4 * A.n_chunk) + 4 * kc + colq] = lc[h];
+                }
             }
         }
     }
     S::teardown(c);
+}
+
+// Flow-only variant: joins the partial statistics of every proxy row and adds up, per query head, the share of each
+// row's attention that lands on the other modality (Eq. 7 over the rows of this call).  One warp per query head.
+__global__ void flow_combine_kernel(const float2 *row_part, const float *row_cross, int n_part, int G, int W, int Hkv, int n_heads,
+                                    float *cross_mass) {
+    const int head = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (head >= n_heads) return;                                         // head = (u * Hkv + h) * G + g
+    const int uh = head / G, g = head % G;
+    float s = 0.f;
+    for (int a = lane; a < W; a += 32) {
+        const int64_t row = ((int64_t)uh * G * W + g * W + a) * n_part;
+        float mx = kNegBig;
+        for (int c = 0; c < n_part; ++c) mx = fmaxf(mx, row_part[row + c].x);
+        float z = 0.f, zc = 0.f;
+        for (int c = 0; c < n_part; ++c) {
+            const float w = exp2f(row_part[row + c].x - mx);
+            z += row_part[row + c].y * w;
+            zc += row_cross[row + c] * w;
+        }
+        s += z > 0.f ? zc / z : 0.f;
+    }
+    s = warp_sum(s);
+    if (lane == 0) cross_mass[(int64_t)(uh / Hkv) * (Hkv * G) + (uh % Hkv) * G + g] = s;
+}
+
+// Packs the modality map: word w of a unit holds keys 32 w .. 32 w + 31 (bit set = visual; keys past the prompt: 0).
+__global__ void pack_modality_kernel(const uint8_t *modality, int L, int n_words, uint32_t *bits) {
+    const int u = blockIdx.y, w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (w >= n_words) return;
+    const int key = 32 * w + lane;
+    const uint32_t word = __ballot_sync(0xFFFFFFFFu, key < L && modality[(int64_t)u * L + key] != 0);
+    if (lane == 0) bits[(int64_t)u * n_words + w] = word;
 }
 
 // Row constants for pass 2: negc[r] = -(M_r + log2 Z_r) so that exp2(s + negc) is the softmax
