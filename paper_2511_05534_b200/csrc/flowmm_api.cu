@@ -349,7 +349,8 @@ flowmm_status run_layer_flow(const flowmm_params &p, const float *cross_mass, fl
 flowmm_status run_select(const flowmm_params &p, const float *importance, int32_t *retained, int32_t *evicted,
                          cudaStream_t st, const float *cross_mass = nullptr, float *rho = nullptr,
                          int32_t *strategy = nullptr) {
-    const int threads = p.seq_len <= 2048 ? 256 : p.seq_len <= 8192 ? 512 : kSelectThreads;
+    const int few = p.n_units * p.n_kv_heads < 2 * tc::sm_count();       // few heads: more threads per head
+    const int threads = few ? (p.seq_len <= 512 ? 256 : kSelectThreads) : p.seq_len <= 2048 ? 256 : p.seq_len <= 8192 ? 512 : kSelectThreads;
     SelectFlow f;
     f.cross_mass = cross_mass; f.rho = rho; f.strategy = strategy; f.Hq = p.n_q_heads; f.Hkv = p.n_kv_heads;
     f.theta = p.theta; f.flow_mode = p.flow_mode;
@@ -375,7 +376,9 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     g.tau_eff = tau_effective(p);
     for (int i = 0; i < 3; ++i) g.ks[i] = p.k_stride[i];
     g.copy_here = y.c_tot <= 256;
-    match_prepare_kernel<<<UH, 256, 0, st>>>(g);
+    // few heads: a head's lists are walked by more threads, the GPU is not full either way
+    const int prep_threads = UH >= 4 * tc::sm_count() ? 256 : UH >= 2 * tc::sm_count() ? 512 : 1024;
+    match_prepare_kernel<<<UH, prep_threads, 0, st>>>(g);
     FLOWMM_LAUNCHED("match_prepare");
     if (!g.copy_here) {
         match_gather_kernel<<<dim3((y.c_tot + 63) / 64, UH), 256, 0, st>>>(g);

@@ -63,8 +63,8 @@ __device__ __forceinline__ void match_gather_rows(const MatchPrepArgs &A, int uh
     }
 }
 
-// grid = U*Hkv, block = 256.
-__global__ void __launch_bounds__(256) match_prepare_kernel(const MatchPrepArgs A) {
+// grid = U*Hkv, block = 256 to 1024 (a multiple of 32).
+__global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs A) {
     __shared__ int scratch[33];
     __shared__ int s_ntext;
     const int tid = threadIdx.x, uh = blockIdx.x, u = uh / A.Hkv, h = uh % A.Hkv;
