@@ -66,7 +66,17 @@ __device__ __forceinline__ float warp_sum(float v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
     return v;
 }
+
+
 __device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
+
+// Sum of one head's partial masses: lanes take the parts with a stride of 32, then a shuffle
+// tree; the order is fixed, so every caller gets the same bits.  Call with the whole warp.
+__device__ __forceinline__ float head_mass(const float *parts, int n_chunk) {
+    float s = 0.f;
+    for (int c = lane_id(); c < n_chunk; c += 32) s += parts[c];
+    return warp_sum(s);
+}
 __device__ __forceinline__ uint32_t lanemask_lt() {
     uint32_t m;
     asm volatile("mov.u32 %0, %%lanemask_lt;" : "=r"(m));

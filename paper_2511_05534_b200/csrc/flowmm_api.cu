@@ -347,12 +347,12 @@ flowmm_status run_layer_flow(const flowmm_params &p, const float *cross_mass, fl
 
 // cross_mass != nullptr: the launch also applies Eq. 6 and the theta rule to the final masses (rho may be nullptr)
 flowmm_status run_select(const flowmm_params &p, const float *importance, int32_t *retained, int32_t *evicted,
-                         cudaStream_t st, const float *cross_mass = nullptr, float *rho = nullptr,
-                         int32_t *strategy = nullptr) {
+                         cudaStream_t st, float *cross_mass = nullptr, float *rho = nullptr,
+                         int32_t *strategy = nullptr, const float *cross_part = nullptr, int n_parts = 0) {
     const int few = p.n_units * p.n_kv_heads < 2 * tc::sm_count();       // few heads: more threads per head
     const int threads = few ? (p.seq_len <= 512 ? 256 : kSelectThreads) : p.seq_len <= 2048 ? 256 : p.seq_len <= 8192 ? 512 : kSelectThreads;
     SelectFlow f;
-    f.cross_mass = cross_mass; f.rho = rho; f.strategy = strategy; f.Hq = p.n_q_heads; f.Hkv = p.n_kv_heads;
+    f.cross_part = cross_part; f.n_parts = n_parts; f.cross_mass = cross_mass; f.rho = rho; f.strategy = strategy; f.Hq = p.n_q_heads; f.Hkv = p.n_kv_heads;
     f.theta = p.theta; f.flow_mode = p.flow_mode;
     select_topb_kernel<<<p.n_units * p.n_kv_heads, threads, 0, st>>>(importance, p.seq_len, p.n_keep, p.window,
                                                                            p.keep_window, retained, evicted, f);
@@ -652,16 +652,9 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
     float *cross_mass = at<float>(ws, y.cross_mass);
     int n_parts = 0;
     FLOWMM_TRY(run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, st, &n_parts));
-    bool flow_in_select = false;
-    if (n_parts == 0) {
-        flow_in_select = true;               // the masses are final: Eq. 6 and the theta rule ride along with the selection
-    } else {
-        flow_from_parts_kernel<<<p->n_units, 256, 0, st>>>(at<float>(ws, y.cross_part), n_parts, p->n_q_heads, p->window,
-                                                           p->theta, p->flow_mode, cross_mass, rho, strategy);
-        FLOWMM_LAUNCHED("flow_from_parts");
-    }
-    if (flow_in_select) FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st, cross_mass, rho, strategy));
-    else FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st));
+    // Eq. 6 and the theta rule ride along with the selection launch (which first adds up the partial masses, if any)
+    FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st, cross_mass, rho, strategy,
+                          n_parts > 0 ? at<float>(ws, y.cross_part) : nullptr, n_parts));
     // when both the short-list matching kernel and the tensor-core merge apply, the former writes the latter's table
     const bool map_in_match = p->seq_len > p->n_keep && use_tc(*p) && y.c_tot <= mst::kMaxCols && merge_is_tc(*p);
     FLOWMM_TRY(run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws, st,

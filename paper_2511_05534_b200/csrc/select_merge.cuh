@@ -20,7 +20,9 @@ __device__ __forceinline__ uint32_t select_key(float v, bool forced) {
 // Eq. 6 and the theta rule riding along with the selection (cross_mass == nullptr: not asked for): the block of a
 // unit's first KV head applies them, one thread, same arithmetic as layer_flow_kernel.
 struct SelectFlow {
-    const float *cross_mass;     // [U, Hq] final per-head masses
+    const float *cross_part;     // nullptr, or [U * Hq, n_parts] partial masses that are first added up into cross_mass
+    int n_parts;
+    float *cross_mass;           // [U, Hq] per-head masses (read; written first when cross_part is given)
     float *rho;                  // [U] or nullptr
     int *strategy;               // [U]
     int Hq, Hkv;
@@ -40,6 +42,15 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
     int *ret = retained + (int64_t)blockIdx.x * B;
     int *evi = evicted + (int64_t)blockIdx.x * (L - B);
     const int first_forced = keep_window ? L - W : L;
+    if (F.cross_part && blockIdx.x % F.Hkv == 0) {                   // (the same for every thread of the block)
+        const int u = blockIdx.x / F.Hkv;
+        for (int g = tid >> 5; g < F.Hq; g += nthreads >> 5) {      // same sums in the same order as cross_mass_reduce
+            const int64_t i = (int64_t)u * F.Hq + g;
+            const float s = head_mass(F.cross_part + i * F.n_parts, F.n_parts);
+            if (lane == 0) F.cross_mass[i] = s;
+        }
+        __syncthreads();
+    }
     if (F.cross_mass && blockIdx.x % F.Hkv == 0 && tid == nthreads - 1) {
         const int u = blockIdx.x / F.Hkv;
         float s = 0.f;

@@ -238,14 +238,6 @@ __global__ void __launch_bounds__(kSimtThreads) score_colsum_simt(const ScoreArg
     }
 }
 
-// Sum of one head's partial masses: lanes take the parts with a stride of 32, then a shuffle
-// tree; the order is fixed, so every caller gets the same bits.  Call with the whole warp.
-__device__ __forceinline__ float head_mass(const float *parts, int n_chunk) {
-    float s = 0.f;
-    for (int c = lane_id(); c < n_chunk; c += 32) s += parts[c];
-    return warp_sum(s);
-}
-
 // cross_mass[u, g] = sum of the per-chunk partial masses; one warp per head.
 __global__ void cross_mass_reduce(const float *cross_part, int n_chunk, int n, float *cross_mass) {
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -264,26 +256,6 @@ __global__ void layer_flow_kernel(const float *cross_mass, int U, int Hq, int W,
     const float r = s / (float)Hq;
     if (rho) rho[u] = r;
     strategy[u] = flow_mode == 1 ? 0 : flow_mode == 2 ? 1 : ((r > theta) != (flow_mode == 3) ? 1 : 0);
-}
-
-// cross_mass_reduce and layer_flow_kernel in one launch (same sums in the same order): one block
-// per unit, one warp per query head, thread 0 then applies Eq. 6 and the theta rule.
-__global__ void flow_from_parts_kernel(const float *cross_part, int n_chunk, int Hq, int W, float theta, int flow_mode,
-                                       float *cross_mass, float *rho, int *strategy) {
-    const int u = blockIdx.x;
-    for (int g = threadIdx.x >> 5; g < Hq; g += blockDim.x >> 5) {
-        const int64_t i = (int64_t)u * Hq + g;
-        const float s = head_mass(cross_part + i * n_chunk, n_chunk);
-        if (lane_id() == 0) cross_mass[i] = s;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float s = 0.f;
-        for (int g = 0; g < Hq; ++g) s += cross_mass[(int64_t)u * Hq + g] / (float)W;   // a head's total mass is W
-        const float r = s / (float)Hq;
-        if (rho) rho[u] = r;
-        strategy[u] = flow_mode == 1 ? 0 : flow_mode == 2 ? 1 : ((r > theta) != (flow_mode == 3) ? 1 : 0);
-    }
 }
 
 // Full-prefill flow: per-head masses of the query tiles added up in tile order, then Eq. 6 over all L rows
