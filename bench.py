@@ -159,7 +159,7 @@ KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
     "score_stats_simt": "score_stats", "score_stats_tc": "score_stats", "score_fused_tc": "score_colsum",
     "score_colsum_simt": "score_colsum", "score_colsum_tc": "score_colsum",
     "inv_norm": "inv_norm", "match_simt": "match", "match_tc": "match", "match_small_tc": "match", "merge_pieces": "merge_pieces",
-    "merge_tc": "merge_pieces",
+    "merge_tc": "merge_pieces", "merge_staged": "merge_pieces",
     "select_topb": "select_topb", "build_csr": "build_csr",
 }
 

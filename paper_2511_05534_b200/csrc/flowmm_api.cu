@@ -12,6 +12,7 @@
 #include "decode.cuh"
 #include "decode_tc.cuh"
 #include "match_small_tc.cuh"
+#include "merge_staged.cuh"
 #include "merge_tc.cuh"
 #include "score_fused_tc.cuh"
 #include "match_tc.cuh"
@@ -530,7 +531,15 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
     if (total_pieces > 0xFFFF0000ll) return FLOWMM_ERR_SHAPE;           // the piece table is indexed with 32 bits
     const int64_t want_blocks = (total_pieces + 7) / 8;
     const int gp = (int)(want_blocks < 2 * tc::sm_count() ? want_blocks : 2 * tc::sm_count());   // persistent warps
-    if (p.dtype == FLOWMM_BF16) {
+    if (p.dtype == FLOWMM_BF16 && p.head_dim == 128 && E > 0 && p.path != FLOWMM_PATH_SIMT) {
+        // rows of 256 bytes: member rows staged through shared memory by asynchronous copies, three CTAs per SM
+        if (cudaFuncSetAttribute(mstg::merge_staged_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)mstg::kSmemBytes) != cudaSuccess)
+            return FLOWMM_ERR_CUDA;
+        const int gs = (int)(want_blocks < 3 * tc::sm_count() ? want_blocks : 3 * tc::sm_count());
+        mstg::merge_staged_kernel<__nv_bfloat16><<<gs, mstg::kThreads, mstg::kSmemBytes, st>>>(m, UH, at<int>(ws, y.merge_status));
+        FLOWMM_LAUNCHED("merge_staged");
+    } else if (p.dtype == FLOWMM_BF16) {
         merge_pieces_kernel<__nv_bfloat16><<<gp, 256, 0, st>>>(m, UH);
         FLOWMM_LAUNCHED("merge_pieces");
     } else {
