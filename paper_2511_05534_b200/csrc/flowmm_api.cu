@@ -537,7 +537,8 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
                                  (int)mstg::kSmemBytes) != cudaSuccess)
             return FLOWMM_ERR_CUDA;
         const int gs = (int)(want_blocks < 3 * tc::sm_count() ? want_blocks : 3 * tc::sm_count());
-        mstg::merge_staged_kernel<__nv_bfloat16><<<gs, mstg::kThreads, mstg::kSmemBytes, st>>>(m, UH, at<int>(ws, y.merge_status));
+        mstg::merge_staged_kernel<__nv_bfloat16><<<gs, mstg::kThreads, mstg::kSmemBytes, st>>>(
+            m, UH, at<int>(ws, y.merge_status), make_fastdiv((uint32_t)m.max_pieces), make_fastdiv((uint32_t)p.n_kv_heads));
         FLOWMM_LAUNCHED("merge_staged");
     } else if (p.dtype == FLOWMM_BF16) {
         merge_pieces_kernel<__nv_bfloat16><<<gp, 256, 0, st>>>(m, UH);

@@ -24,7 +24,8 @@ constexpr uint32_t kWarpBytes = 2 * kBufBytes;
 constexpr uint32_t kSmemBytes = (kThreads / 32) * kWarpBytes + (kThreads / 32) * 16 + 16;
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeArgs A, int n_uh, int *status) {
+__global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeArgs A, int n_uh, int *status,
+                                                                   const FastDiv by_pieces, const FastDiv by_hkv) {
     static_assert(sizeof(T) * 128 == 256 || sizeof(T) * 64 == 256, "rows of 256 bytes");
     constexpr int V = Elem<T>::kVec;
     extern __shared__ __align__(128) uint8_t mstg_smem[];
@@ -51,7 +52,7 @@ __global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeAr
     auto fetch_members = [&](unsigned g, Piece &pc) {        // needs pc.d
         pc.tok_lo = pc.tok_hi = pc.r = 0; pc.w_lo = pc.w_hi = 0.f;
         if (pc.d.z < 0) return;
-        const int64_t uh = g / (unsigned)A.max_pieces;
+        const int64_t uh = by_pieces.div(g);
         if (pc.d.z > 0) {
             const int *mt = A.mem_tok + uh * A.E + pc.d.y;
             const float *mw = A.mem_w + uh * A.E + pc.d.y;
@@ -74,8 +75,19 @@ __global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeAr
     };
     // Starts the copies of batch `b` of a piece into buffer `j & 1` (j = batches this warp has started so far):
     // row slot 0 = the pivot (first batch of a single-piece slot only), slots 1.. = members 8 b .. 8 b + 7.
+    // this lane's source rows (K for lanes 0-15, V for 16-31) and output rows of one (unit, head), kept until the head changes
+    int src_uh = -1, dst_uh = -1;
+    const T *src_base = nullptr;
+    T *dst_base = nullptr;
+    const int64_t tstride = is_v ? A.vs[2] : A.ks[2], ostride = is_v ? A.vos[2] : A.kos[2];
     auto issue = [&](const Piece &pc, unsigned g, int b, int j) {
-        const int uh = (int)(g / (unsigned)A.max_pieces), u = uh / A.Hkv, h = uh % A.Hkv;
+        const int uh = (int)by_pieces.div(g);
+        if (uh != src_uh) {
+            const int u = (int)by_hkv.div(uh), h = uh - u * A.Hkv;
+            src_base = is_v ? static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1]
+                            : static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
+            src_uh = uh;
+        }
         const int n_mem = min(kBatch, pc.d.z - b * kBatch);
         const bool pivot = b == 0 && pc.d.w < 0;
         const uint32_t buf = bufs + (j & 1) * kBufBytes, bar = bar0 + (j & 1) * 8;
@@ -84,9 +96,6 @@ __global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeAr
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         if (lane == 0) tc::mbar_expect_tx(bar, (uint32_t)(n_mem + (pivot ? 1 : 0)) * kRowBytes);
         __syncwarp();
-        const T *base = is_v ? static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1]
-                             : static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
-        const int64_t tstride = is_v ? A.vs[2] : A.ks[2];
         // lane l < 16 copies a row's K part, lane 16 + l its V part: rows l = 0 .. 8 (0 = pivot)
         const int rowslot = lane & 15;
         const int t = b * kBatch + rowslot - 1;               // member index of this lane's row
@@ -95,7 +104,7 @@ __global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeAr
         int tok = t < 32 ? tok_a : tok_b;
         bool go = rowslot >= 1 && rowslot <= n_mem;
         if (rowslot == 0) { tok = pc.r; go = pivot; }
-        if (go) tc::bulk_load(buf + rowslot * kRowBytes + (is_v ? 256u : 0u), base + (int64_t)tok * tstride, 256u, bar);
+        if (go) tc::bulk_load(buf + rowslot * kRowBytes + (is_v ? 256u : 0u), src_base + (int64_t)tok * tstride, 256u, bar);
     };
 
     unsigned g = next_piece(), g_nxt = next_piece();
@@ -113,7 +122,7 @@ __global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeAr
         const int slot = cur.d.x, count = cur.d.z, part = cur.d.w;
         bool next_started = false;
         if (count >= 0) {
-            const int uh = (int)(g / (unsigned)A.max_pieces), u = uh / A.Hkv, h = uh % A.Hkv;
+            const int uh = (int)by_pieces.div(g);
             const int nb = count > 0 ? (count + kBatch - 1) / kBatch : 1;
             if (!started) { issue(cur, g, 0, j); ++j; }
             float acc[V];
@@ -150,8 +159,13 @@ __global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeAr
             }
             if (!ok) break;
             if (part < 0) {
-                T *dst = is_v ? static_cast<T *>(A.v_out) + u * A.vos[0] + h * A.vos[1] + (int64_t)slot * A.vos[2]
-                              : static_cast<T *>(A.k_out) + u * A.kos[0] + h * A.kos[1] + (int64_t)slot * A.kos[2];
+                if (uh != dst_uh) {
+                    const int u = (int)by_hkv.div(uh), h = uh - u * A.Hkv;
+                    dst_base = is_v ? static_cast<T *>(A.v_out) + u * A.vos[0] + h * A.vos[1]
+                                    : static_cast<T *>(A.k_out) + u * A.kos[0] + h * A.kos[1];
+                    dst_uh = uh;
+                }
+                T *dst = dst_base + (int64_t)slot * ostride;
                 if (count == 0) {
                     *reinterpret_cast<uint4 *>(dst + c0) = xr;       // nothing merged in: the pivot row, bit for bit
                 } else {
