@@ -419,6 +419,7 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     a.cand_scale = g.cand_scale; a.modality = mod; a.tile_mod = g.tile_mod;
     a.match = match; a.match_sim = match_sim; a.status = at<int>(ws, y.status);
     a.Hkv = p.n_kv_heads; a.L = p.seq_len; a.E = E; a.Ctot = y.c_tot; a.n_rt = y.n_rt; a.n_items = UH * y.n_rt;
+    a.by_nrt = make_fastdiv((uint32_t)y.n_rt); a.by_hkv = make_fastdiv((uint32_t)p.n_kv_heads);
     if (cudaFuncSetAttribute(match_tc_kernel<tcs::Big>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tcs::Big::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(match_tc_kernel<tcs::Small>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -136,6 +136,7 @@ struct MatchTcArgs {
     float *match_sim;
     int *status;
     int Hkv, L, E, Ctot, n_rt, n_items;
+    FastDiv by_nrt, by_hkv;      // exact division of item numbers by n_rt and of head numbers by Hkv
 };
 
 struct MatchItem {
@@ -151,7 +152,7 @@ struct MatchRaw { int n_text, n_vis, strategy, tile_mod; };
 __device__ __forceinline__ MatchRaw match_raw(const MatchTcArgs &A, int item) {
     MatchRaw r = {0, 0, 1, 0};
     if (item >= A.n_items) return r;
-    const int uh = item / A.n_rt, rt = item % A.n_rt, u = uh / A.Hkv;
+    const int uh = (int)A.by_nrt.div(item), rt = item - uh * A.n_rt, u = (int)A.by_hkv.div(uh);
     r.n_text = A.cand_count[2 * uh]; r.n_vis = A.cand_count[2 * uh + 1];
     r.strategy = A.strategy[u];
     r.tile_mod = A.tile_mod[(int64_t)u * A.n_rt + rt];
@@ -164,8 +165,8 @@ template <class S>
 __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item, const MatchRaw &raw) {
     constexpr int kMtCols = S::kCols;        // candidates per column tile
     MatchItem p;
-    p.uh = item / A.n_rt; p.rt = item % A.n_rt;
-    p.u = p.uh / A.Hkv; p.h = p.uh % A.Hkv;
+    p.uh = (int)A.by_nrt.div(item); p.rt = item - p.uh * A.n_rt;
+    p.u = (int)A.by_hkv.div(p.uh); p.h = p.uh - p.u * A.Hkv;
     p.n_text = raw.n_text; p.n_vis = raw.n_vis;
     p.t0 = (p.n_text + 31) & ~31;
     p.intra = raw.strategy == 0;
@@ -213,14 +214,14 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         bool ok = true;
         // what an item needs from global memory is fetched one item ahead: its plan values, the token's
         // modality and its place in the non-pivot list
-        auto token_of = [&](int item) { return (item % A.n_rt) * kMtItemRows + c.group * kMtRows + row; };
+        auto token_of = [&](int item) { return (item - (int)A.by_nrt.div(item) * A.n_rt) * kMtItemRows + c.group * kMtRows + row; };
         auto fetch_mod = [&](int item) -> int {
             const int token = token_of(item);
-            return item < A.n_items && token < A.L ? A.modality[(int64_t)(item / A.n_rt / A.Hkv) * A.L + token] : 0;
+            return item < A.n_items && token < A.L ? A.modality[(int64_t)A.by_hkv.div(A.by_nrt.div(item)) * A.L + token] : 0;
         };
         auto fetch_rank = [&](int item) -> int {
             const int token = token_of(item);
-            return item < A.n_items && token < A.L ? A.rank[(int64_t)(item / A.n_rt) * A.L + token] : -1;
+            return item < A.n_items && token < A.L ? A.rank[(int64_t)A.by_nrt.div(item) * A.L + token] : -1;
         };
         MatchRaw raw_next = match_raw(A, blockIdx.x);
         int mod_next = fetch_mod(blockIdx.x), rank_next = fetch_rank(blockIdx.x);
