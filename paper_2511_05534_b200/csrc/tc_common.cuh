@@ -46,13 +46,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// The same with a suspend-time hint: the thread may sleep up to `ns` nanoseconds inside the instruction and
+// wakes when the phase completes, so a long wait costs few issue slots and few shared-memory requests.
+__device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+constexpr uint32_t kWaitSuspendNs = 2000;
+
 // Bounded wait.  `abort_flag` (shared memory) is raised by whichever thread of the CTA runs out
 // of time first; every other waiter sees it and gives up too.  Returns false on give-up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status_word) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
     for (uint32_t spins = 1;; ++spins) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_for(bar, parity, kWaitSuspendNs)) return true;
+        if ((spins & 15u) != 0) continue;
         if (*abort_flag) return false;
         if ((spins & 1023u) == 0) {
             const unsigned long long now = global_timer_ns();
