@@ -152,7 +152,7 @@ def kernel_model(wl, B, dsize):
 # the whole stack of the workload (profiles/ has the commands); None where no capture was taken.
 NCU_TRAFFIC = {
     ("cfg2", 100): {"score_fused_tc": 181.3e6, "match_small_tc": 203.0e6, "merge_tc": 365.1e6},
-    ("cfg4", 200): {"match_tc": 305.4e6, "score_stats_tc": 261.4e6, "score_colsum_tc": 262.4e6, "merge_pieces": 580.5e6},
+    ("cfg4", 200): {"match_tc": 305.4e6, "score_stats_tc": 261.4e6, "score_colsum_tc": 262.4e6, "merge_staged": 578.8e6},
 }
 
 KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
