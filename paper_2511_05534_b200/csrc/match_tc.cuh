@@ -315,7 +315,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 }
             }
             // (after a wait that ran out the results are garbage, but the two meeting points below are still
-            // kept so that the partner warp is never left waiting; the loop ends right after them)
+            // kept so that the partner warp is never left waiting; the first one tells both warps, and the loop
+            // ends for both right after them)
             // this warp's result for the row: similarity (still times the row's norm) and pivot slot
             int slot = -1;
             if (best_cc >= 0 && ok) {
@@ -332,7 +333,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             }
             // the upper column half hands its result to the lower one, which owns the row's output
             if (c.colhalf == 1) tc::sts128(wrow, best, __int_as_float(slot), 0.f, 0.f);
-            S::pair_sync(c);
+            ok = !S::pair_meet(c, !ok);                            // (both warps of a row go on, or neither)
             if (c.colhalf == 0 && ok) {
                 const float4 other = tc::lds128(prow);
                 if (other.x > best) { best = other.x; slot = __float_as_int(other.y); }    // a tie stays with the lower columns

@@ -360,7 +360,7 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
             // the two column halves of a key meet: the upper one hands its partial sum over (kept even after a
             // wait ran out, so that the partner warp is never left waiting)
             if (c.colhalf == 1) tc::sts32(xch, imp);
-            S::pair_sync(c);
+            ok = !S::pair_meet(c, !ok);                            // (both warps of a key go on, or neither)
             if (c.colhalf == 0 && ok && key < A.L) A.importance[(int64_t)uh * A.L + key] = (imp + tc::lds32(pxch)) / (float)A.G;   // group mean
             S::pair_sync(c);
         }

@@ -299,6 +299,20 @@ struct Skel {
             f(ch, a);
         }
     }
+    // The same meeting point with a vote: returns whether either warp has given up on a wait, so that both leave
+    // the item loop together and neither is left alone at the next meeting.
+    static __device__ __forceinline__ bool pair_meet(const Ctx &c, bool gave_up) {
+        uint32_t any;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.u32 q, %1, 0;\n\t"
+            "barrier.cta.red.or.pred p, %2, 64, q;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(any)
+            : "r"((uint32_t)gave_up), "r"(1 + c.group * 4 + c.quarter)
+            : "memory");
+        return any != 0;
+    }
     // Meeting point of the two warps that share rows (same half, same lanes, other columns).
     static __device__ __forceinline__ void pair_sync(const Ctx &c) {
         asm volatile("bar.sync %0, 64;" ::"r"(1 + c.group * 4 + c.quarter) : "memory");
