@@ -148,11 +148,11 @@ def kernel_model(wl, B, dsize):
     return m
 
 
-# DRAM bytes (read + write) of one launch from `ncu --set full` captures of the committed kernels on
-# the whole stack of the workload (profiles/ has the commands); None where no capture was taken.
+# DRAM bytes (read + write) of one launch from ncu captures of the committed kernels on the whole stack of the
+# workload (profiles/dram_traffic_cfg2_cfg4.md has the commands and the counters); None where no capture was taken.
 NCU_TRAFFIC = {
-    ("cfg2", 100): {"score_fused_tc": 181.3e6, "match_small_tc": 203.0e6, "merge_tc": 365.1e6},
-    ("cfg4", 200): {"match_tc": 305.4e6, "score_stats_tc": 261.4e6, "score_colsum_tc": 262.4e6, "merge_staged": 578.8e6},
+    ("cfg2", 100): {"score_fused_tc": 180.3e6, "match_small_tc": 201.1e6, "merge_tc": 361.7e6},
+    ("cfg4", 200): {"match_tc": 302.9e6, "score_stats_tc": 260.8e6, "score_colsum_tc": 258.5e6, "merge_staged": 575.7e6},
 }
 
 KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
