@@ -303,7 +303,8 @@ def run_ours(args):
                 torch.cuda.synchronize()
                 for i in range(n_sets):
                     g = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(g, stream=side):
+                    # (thread_local: calls of other threads, a process group's watchdog for one, do not disturb the capture)
+                    with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
                         step(i)
                     graphs.append(g)
             torch.cuda.synchronize()
