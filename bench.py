@@ -1,11 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the FlowMM per-layer KV-cache compression on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--permille 100]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--permille 50]
     python bench.py --impl reference ...       # the fp64 CPU oracle as the reference arm
 
 A step is one flowmm_compress_layer call over every (layer, sequence) unit of
-the workload's stack.  The metric is context tokens compressed per second per
+the workload's stack (default: the long-context workload cfg5, 80 layers x 4
+sequences of 33 792 tokens, the largest one that fits a GPU).  The metric is context tokens compressed per second per
 layer: n_seqs * L * n_layers / step time, summed over GPUs (each GPU compresses
 its own sequences; units are independent, so there is no collective on the
 data path).  Prints one JSON line.
@@ -31,17 +32,21 @@ UNIT = "tokens/s/layer"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--permille", type=int, default=0,
                     help="retention budget in 1/1000 of the context (0: 100 if the workload lists it, else its first)")
     ap.add_argument("--layers", type=int, default=0, help="use only the first N layers (0 = the whole stack)")
     ap.add_argument("--path", default="auto", choices=["auto", "simt"])
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets held on the device (0 = automatic)")
-    ap.add_argument("--launch", choices=["graph", "plain"], default="graph",
-                    help="timed steps: replay of CUDA graphs captured from the call (default) or the plain calls")
+    ap.add_argument("--launch", choices=["graph", "plain"], default="plain",
+                    help="plain: the timed steps are the library calls (default); graph: the steps are also replayed "
+                         "from CUDA graphs captured from the call and that time is reported beside the value")
+    ap.add_argument("--cpu-seconds", type=float, default=20.0, help="CPU time the oracle baseline leg may spend")
+    ap.add_argument("--reference-seconds", type=float, default=150.0,
+                    help="--impl reference: wall time its warm-up and timed steps may spend together")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="skip the decode-attention timing over the caches")
     ap.add_argument("--cpu-baseline-units", type=int, default=0)
@@ -68,6 +73,8 @@ class ClockSampler:
         self._stop = False
         self._thread = None
         self._err = None
+        self._ready = None
+        self._mark = 0
 
     def _run(self):
         try:
@@ -90,21 +97,32 @@ class ClockSampler:
                 for bit, name in table.items():
                     if bits & bit:
                         self.reasons.add(name)
+                self._ready.set()
                 time.sleep(0.002)
         except Exception as exc:            # NVML missing or refused: report it, do not fail the run
             self._err = repr(exc)
+            self._ready.set()
 
     def start(self):
+        """Starts the helper thread and returns once its first sample is in (NVML is up by then)."""
         import threading
+        self._ready = threading.Event()
         self._thread = threading.Thread(target=self._run, daemon=True)
         self._thread.start()
+        self._ready.wait(timeout=30)
+
+    def mark(self):
+        """Samples taken before this call (warm-up, idle) are left out of the summary."""
+        self._mark = len(self.samples)
+        self.reasons.clear()
 
     def stop(self):
         self._stop = True
         if self._thread is not None:
             self._thread.join(timeout=5)
-        out = {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.sm_max,
-               "samples": len(self.samples), "reasons": sorted(self.reasons)}
+        timed = self.samples[self._mark:]
+        out = {"sm_mhz": statistics.median(timed) if timed else None, "sm_max_mhz": self.sm_max,
+               "samples": len(timed), "reasons": sorted(self.reasons)}
         if self._err:
             out["error"] = self._err
         return out
@@ -150,12 +168,32 @@ def kernel_model(wl, B, dsize):
     return m
 
 
-# DRAM bytes (read + write) of one launch from ncu captures of the committed kernels on the whole stack of the
-# workload (profiles/dram_traffic_cfg2_cfg4.md has the commands and the counters); None where no capture was taken.
-NCU_TRAFFIC = {
-    ("cfg2", 100): {"score_fused_tc": 180.3e6, "match_small_tc": 201.1e6, "merge_tc": 361.7e6},
-    ("cfg4", 200): {"match_tc": 302.9e6, "score_stats_tc": 260.8e6, "score_colsum_tc": 258.5e6, "merge_staged": 575.7e6},
-}
+def csrc_digest():
+    """sha256 over the CUDA sources and the public header, in name order: identifies the kernels as built."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2511_05534_b200", "csrc")
+    for path in sorted(os.path.join(csrc, f) for f in os.listdir(csrc)) + [os.path.join(ROOT, "include", "flowmm.h")]:
+        h.update(os.path.basename(path).encode())
+        h.update(open(path, "rb").read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload, permille, units, kernel):
+    """DRAM bytes (read + write) of one launch of `kernel` from the committed table of ncu captures
+    (paper_2511_05534_b200/ncu_traffic.json; the summaries under profiles/ give the commands).  An entry is
+    per unit of its workload and budget, taken on a small case, and scaled by the units of this call (traffic
+    of these kernels grows in proportion to the units).  None when there is no entry, or when the sources have
+    changed since the counters were taken."""
+    path = os.path.join(ROOT, "paper_2511_05534_b200", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return None
+    table = json.load(open(path))
+    if table.get("csrc_digest") != csrc_digest():
+        return None
+    per_unit = table.get("bytes_per_unit", {}).get("%s@%d" % (workload, permille), {}).get(kernel)
+    return None if per_unit is None else per_unit * units
+
 
 KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
     "score_stats_simt": "score_stats", "score_stats_tc": "score_stats", "score_fused_tc": "score_colsum",
@@ -166,44 +204,74 @@ KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
 }
 
 
+# Share of a scoring kernel's exponentials that it evaluates as a polynomial on the FMA pipe (the kernels' own
+# constants: score_tc.cuh); the rest goes through the exp2 unit.
+EXP_FMA_SHARE = {"score_stats_tc": 0.25, "score_colsum_tc": 0.0}
+
+
 def model_for(name, model):
     return model.get(KERNEL_MODEL.get(name, ""), (0.0, 0.0))
 
 
-def run_reference(args):
-    """The oracle as the reference arm: each step compresses a bounded sample of the stack."""
-    import numpy as np
+def _oracle_sample(wl, permille, n_units):
+    """A bounded sample of the workload for the oracle: `n_units` layers spread over the stack, sequence 0."""
     from oracle import flowmm_oracle as O
-    from paper_2511_05534_b200 import configs, inputs
+    from paper_2511_05534_b200 import inputs
+    B = wl.n_keep(permille)
+    n_units = max(1, min(n_units, wl.n_layers))
+    layers = sorted(set(int(round(i * (wl.n_layers - 1) / max(1, n_units - 1))) for i in range(n_units)))
+    if n_units == 1:
+        layers = [wl.n_layers // 2]
+    units = [(l, 0) for l in layers]
+    data = inputs.make_units(wl, units)
+    p = O.OracleParams(len(units), wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.seq_len, wl.window, B,
+                       theta=wl.theta, tau=wl.tau_rel, tau_mode=O.TAU_REL)
+    return p, data, layers
+
+
+def _oracle_units_per_step(wl):
+    """How many layers of the stack one oracle step covers, by context length (a step of seconds, not minutes)."""
+    return 8 if wl.seq_len <= 1024 else (4 if wl.seq_len <= 4096 else (2 if wl.seq_len <= 16384 else 1))
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step compresses a bounded sample of the stack; warm-up and timed
+    steps together are held to --reference-seconds of wall time (fewer steps are timed if they would not fit,
+    and the line says how many were)."""
+    from oracle import flowmm_oracle as O
+    from paper_2511_05534_b200 import configs
 
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     wl = configs.get(args.workload)
     B = wl.n_keep(args.permille)
-    n_sample = min(wl.n_layers, 8 if wl.seq_len <= 1024 else 2)
-    layers = sorted(set(int(round(i * (wl.n_layers - 1) / max(1, n_sample - 1))) for i in range(n_sample)))
-    if wl.seq_len > 4096:
-        layers = layers[:1]
-    units = [(l, 0) for l in layers]
-    data = inputs.make_units(wl, units)
-    p = O.OracleParams(len(units), wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.seq_len, wl.window, B,
-                       theta=wl.theta, tau=wl.tau_rel, tau_mode=O.TAU_REL)
     O.build()
-    for _ in range(args.warmup):
+    p, data, layers = _oracle_sample(wl, args.permille, _oracle_units_per_step(wl))
+
+    def one():
+        t0 = time.perf_counter()
         O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
-    steps = max(1, args.steps)
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
-    dt = (time.perf_counter() - t0) / steps
-    value = wl.seq_len * len(units) / dt
-    sample = "layers %s of the %s stack, one sequence, per step; %d timed steps" % (layers, wl.name, steps)
+        return time.perf_counter() - t0
+
+    budget = max(1.0, args.reference_seconds)
+    spent, warm = 0.0, 0
+    while warm < max(1, args.warmup) and (warm == 0 or spent + spent / warm <= 0.2 * budget):
+        spent += one()
+        warm += 1
+    per_step = spent / warm
+    steps = max(1, min(max(1, args.steps), int((budget - spent) / per_step)))
+    times = [one() for _ in range(steps)]
+    dt = sum(times) / steps
+    value = wl.seq_len * len(layers) / dt
+    sample = ("layers %s of the %s stack, one sequence, per step; %d warm-up and %d timed steps (asked: %d and %d; "
+              "held to %.0f s of wall time)" % (layers, wl.name, warm, steps, args.warmup, args.steps, budget))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "budget_permille": args.permille, "n_keep": B, "sample": sample},
+        "config": {"workload": wl.name, "layers": wl.n_layers, "seqs": wl.n_seqs, "budget_permille": args.permille,
+                   "n_keep": B, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -211,31 +279,25 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def cpu_baseline(wl, permille, n_units):
-    import numpy as np
+def cpu_baseline(wl, permille, n_units, seconds):
+    """The oracle as it stands on the host cores, on a bounded sample: repeated until `seconds` of CPU wall
+    time are spent (at least once, at most 20 times)."""
     from oracle import flowmm_oracle as O
-    from paper_2511_05534_b200 import inputs
 
-    B = wl.n_keep(permille)
     if n_units <= 0:
-        n_units = wl.n_layers if wl.seq_len <= 1024 else (4 if wl.seq_len <= 4096 else 1)
-    n_units = min(n_units, wl.n_layers)
-    layers = sorted(set(int(round(i * (wl.n_layers - 1) / max(1, n_units - 1))) for i in range(n_units)))
-    units = [(l, 0) for l in layers]
-    data = inputs.make_units(wl, units)
-    p = O.OracleParams(len(units), wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.seq_len, wl.window, B,
-                       theta=wl.theta, tau=wl.tau_rel, tau_mode=O.TAU_REL)
+        n_units = wl.n_layers if wl.seq_len <= 1024 else _oracle_units_per_step(wl)
     O.build()
+    p, data, layers = _oracle_sample(wl, permille, n_units)
     reps, t_total = 0, 0.0
-    while t_total < 10.0 and reps < 20:
+    while reps < 20 and (reps == 0 or t_total + t_total / reps <= seconds):
         t0 = time.perf_counter()
         O.compress_layer(p, data["q"], data["k"], data["v"], data["modality"])
         t_total += time.perf_counter() - t0
         reps += 1
     dt = t_total / reps
-    return {"value": wl.seq_len * len(units) / dt, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
-            "sample": "%d layer(s) %s of %s, one sequence, %d repetition(s), %.1f s of CPU time" %
-                      (len(units), layers, wl.name, reps, t_total)}
+    return {"value": wl.seq_len * len(layers) / dt, "unit": UNIT, "cores": O.threads(), "kind": "oracle",
+            "sample": "%d layer(s) %s of the %d-layer %s stack, one of its %d sequence(s), %d repetition(s), %.1f s of CPU "
+                      "wall time" % (len(layers), layers, wl.n_layers, wl.name, wl.n_seqs, reps, t_total)}
 
 
 def run_ours(args):
@@ -287,14 +349,29 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()                          # returns after its first sample: NVML is up before anything is timed
     for i in range(max(3, args.warmup)):
         step(i)
     launches_per_step = F.flowmm_last_launch_count()
     barrier()
-    # The call is stream-ordered and allocation-free: one CUDA graph per input set is captured once and the timed
-    # steps replay them (same kernels, same work; only the host's launch gaps go).  --launch plain times the calls.
-    launch_mode = "plain"
-    plain_step = step
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # the timed region: exactly --steps plain library calls, CUDA events on the launching stream
+    sampler.mark()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    status = F.flowmm_last_device_status(ws)
+    if status != 0:
+        raise RuntimeError("device status: " + F.status_string(status))
+    # Beside it, on request: the same steps replayed from CUDA graphs captured from the call, one per input set
+    # (the call is stream-ordered and allocation-free; same kernels and work, only the host's launch gaps go).
+    graph_ms_step = None
     if args.launch == "graph":
         try:
             graphs, side = [], torch.cuda.Stream(device=dev)
@@ -308,39 +385,24 @@ def run_ours(args):
                         step(i)
                     graphs.append(g)
             torch.cuda.synchronize()
-
-            def step(i):                         # noqa: F811  (the timed loop below replays)
-                graphs[i % n_sets].replay()
-
             for i in range(3):
-                step(i)
-            launch_mode = "cuda graph replay, one graph per input set"
-        except Exception as exc:                 # capture refused: time the plain calls and say so
-            sys.stderr.write("graph capture failed (%s): timing plain launches\n" % exc)
-            step = plain_step
-    barrier()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        step(i)
-    e1.record()
-    barrier()
-    ms_total = e0.elapsed_time(e1)
-    clocks = sampler.stop() if rank == 0 else None
-    status = F.flowmm_last_device_status(ws)
-    if status != 0:
-        raise RuntimeError("device status: " + F.status_string(status))
+                graphs[i % n_sets].replay()
+            barrier()
+            e0.record()
+            for i in range(args.steps):
+                graphs[i % n_sets].replay()
+            e1.record()
+            barrier()
+            graph_ms_step = shard.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+            del graphs
+        except Exception as exc:                 # capture refused: say so, the plain timing stands
+            sys.stderr.write("graph capture failed (%s)\n" % exc)
     ms_total = shard.max_over_ranks(ms_total, dev)
     ms_step = ms_total / args.steps
     tokens_layers = wl.n_seqs * wl.seq_len * n_layers        # tokens x layers compressed per step per GPU
     value = shard.aggregate_throughput(tokens_layers, world, ms_step)
 
     # per-kernel attribution: the same steps again with an event after every kernel
-    if launch_mode != "plain":
-        step = plain_step
     F.flowmm_profile_enable(True)
     per_kernel = {}
     for i in range(args.steps):
@@ -358,6 +420,13 @@ def run_ours(args):
     pairs = match_pair_count(p, tau_eff, diag, m0)
     dense_pairs = float(U) * wl.n_kv_heads * (wl.seq_len - B) * B
     del diag
+    # Three ceilings per kernel: the tensor cores (sustained bf16 peak), HBM, and for the scoring passes the
+    # exp2 unit: one exponential per attention logit and pass, 16 results per clock per SM, at the SM clock
+    # sampled during the timed region, less the share of exponentials the kernel evaluates as a polynomial on
+    # the FMA pipe instead (EXP_FMA_SHARE).  A kernel is measured against the slowest of its ceilings.
+    sm_mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+    exp_peak = 16.0 * torch.cuda.get_device_properties(dev).multi_processor_count * sm_mhz * 1e6   # exponentials / s
+    n_exp_unit = float(wl.n_q_heads) * wl.window * wl.seq_len
     kernels = {}
     for name, times in per_kernel.items():
         avg = sum(times) / len(times)
@@ -365,74 +434,105 @@ def run_ours(args):
         flops, nbytes = flops * U, nbytes * U
         if KERNEL_MODEL.get(name) == "match":
             flops = 2.0 * wl.head_dim * pairs
-        t_tensor = flops / (peaks["bf16_tflops_sustained"] * 1e12) if dt_code == F.BF16 else 0.0
-        t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
-        bound = "tensor" if t_tensor > t_hbm else "hbm"
+        n_exp = n_exp_unit * U * (1.0 - EXP_FMA_SHARE[name]) if name in EXP_FMA_SHARE else 0.0
+        t = {"tensor": flops / (peaks["bf16_tflops_sustained"] * 1e12) if dt_code == F.BF16 else 0.0,
+             "hbm": nbytes / (peaks["hbm_gbs"] * 1e9), "alu": n_exp / exp_peak}
+        bound = max(t, key=lambda b: t[b])
         kernels[name] = {"ms": avg, "bound": bound, "gbs": nbytes / (avg * 1e-3) / 1e9,
-                         "tflops": flops / (avg * 1e-3) / 1e12,
-                         "frac": (t_tensor if bound == "tensor" else t_hbm) / (avg * 1e-3)}
+                         "tflops": flops / (avg * 1e-3) / 1e12, "frac": t[bound] / (avg * 1e-3)}
+        if n_exp > 0:
+            kernels[name].update({"gexp_s": n_exp / (avg * 1e-3) / 1e9, "frac_tensor": t["tensor"] / (avg * 1e-3),
+                                  "frac_exp_unit": t["alu"] / (avg * 1e-3)})
     top = max(kernels, key=lambda n: kernels[n]["ms"])
     tk = kernels[top]
     if tk["bound"] == "tensor":
         roofline = {"kernel": top, "bound": "tensor", "achieved": tk["tflops"], "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": tk["frac"], "traffic": None,
                     "peak_source": peaks["source"] + " (sustained bf16)"}
+    elif tk["bound"] == "alu":
+        roofline = {"kernel": top, "bound": "alu", "achieved": tk["gexp_s"], "peak": exp_peak / 1e9,
+                    "unit": "Gexp2/s", "frac": tk["frac"], "traffic": None, "frac_tensor": tk["frac_tensor"],
+                    "peak_source": "derived: 16 exp2 per clock per SM x %d SMs x %.0f MHz sampled; exponentials the "
+                                   "kernel sends to the FMA pipe (%.0f %%) are not counted" %
+                                   (torch.cuda.get_device_properties(dev).multi_processor_count, sm_mhz,
+                                    100 * EXP_FMA_SHARE[top])}
     else:
         roofline = {"kernel": top, "bound": "hbm", "achieved": tk["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": tk["frac"], "traffic": None, "peak_source": peaks["source"]}
     roofline["launch_ms"] = tk["ms"]
-    if n_layers == wl.n_layers:
-        roofline["traffic"] = NCU_TRAFFIC.get((wl.name, args.permille), {}).get(top)
-    roofline["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)"
+    roofline["traffic"] = ncu_traffic(wl.name, args.permille, U, top)
+    roofline["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, scaled from a small capture by units)"
     roofline["algorithmic_bytes"] = model_for(top, model)[1] * U
+    roofline["share_of_step"] = tk["ms"] / sum(k2["ms"] for k2 in kernels.values())
 
     # end to end: pinned host inputs -> device -> compress -> pinned host result, every step.  Two streams with their
     # own device buffers take the steps alternately, so that one step's result goes back to the host while the next
     # step's inputs come in (the two directions of the host link); every step still moves all of its bytes.
-    hq, hk, hv, hm = (t.cpu().pin_memory() for t in sets[0])
-    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hm))
-    lanes = []
-    for _ in range(2 if bytes_per_set < 8e9 else 1):
-        lanes.append({"s": torch.cuda.Stream(device=dev), "in": [torch.empty_like(t) for t in sets[0]],
-                      "ko": torch.empty_like(k_out), "vo": torch.empty_like(v_out), "ws": F.alloc_workspace(p, dev),
-                      "hko": torch.empty_like(k_out, device="cpu").pin_memory(),
-                      "hvo": torch.empty_like(v_out, device="cpu").pin_memory()})
-    d2h = sum(t.numel() * t.element_size() for t in (lanes[0]["hko"], lanes[0]["hvo"]))
-    e2e_steps = max(4, min(args.steps, 10))
+    def end_to_end():
+        # every rank of the node pins a whole input set: all ranks agree beforehand on whether the host has room
+        import psutil
+        need = sum(t.numel() * t.element_size() for t in sets[0]) + 2 * k_out.numel() * k_out.element_size()
+        fits = torch.tensor([1.0 if psutil.virtual_memory().available > 1.2 * need * world else 0.0], device=dev)
+        if world > 1:
+            dist.all_reduce(fits, op=dist.ReduceOp.MIN)
+        if fits.item() == 0.0:
+            raise MemoryError("host memory cannot hold %d pinned input sets of %.1f GB" % (world, need / 1e9))
+        hq, hk, hv, hm = (t.cpu().pin_memory() for t in sets[0])
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hm))
+        lanes = []
+        for _ in range(2 if bytes_per_set < 8e9 else 1):
+            lanes.append({"s": torch.cuda.Stream(device=dev), "in": [torch.empty_like(t) for t in sets[0]],
+                          "ko": torch.empty_like(k_out), "vo": torch.empty_like(v_out), "ws": F.alloc_workspace(p, dev),
+                          "hko": torch.empty_like(k_out, device="cpu").pin_memory(),
+                          "hvo": torch.empty_like(v_out, device="cpu").pin_memory()})
+        d2h = sum(t.numel() * t.element_size() for t in (lanes[0]["hko"], lanes[0]["hvo"]))
+        e2e_steps = max(4, min(args.steps, 10))
 
-    def e2e_step(i):
-        ln = lanes[i % len(lanes)]
-        with torch.cuda.stream(ln["s"]):
-            for d, h in zip(ln["in"], (hq, hk, hv, hm)):
-                d.copy_(h, non_blocking=True)
-            F.flowmm_compress_layer(p, *ln["in"], ln["ko"], ln["vo"], ln["ws"])
-            ln["hko"].copy_(ln["ko"], non_blocking=True)
-            ln["hvo"].copy_(ln["vo"], non_blocking=True)
+        def e2e_step(i):
+            ln = lanes[i % len(lanes)]
+            with torch.cuda.stream(ln["s"]):
+                for d, h in zip(ln["in"], (hq, hk, hv, hm)):
+                    d.copy_(h, non_blocking=True)
+                F.flowmm_compress_layer(p, *ln["in"], ln["ko"], ln["vo"], ln["ws"])
+                ln["hko"].copy_(ln["ko"], non_blocking=True)
+                ln["hvo"].copy_(ln["vo"], non_blocking=True)
 
-    for i in range(len(lanes)):
-        e2e_step(i)
-    barrier()
-    t_host0 = time.perf_counter()
-    for ln in lanes:
-        ln["s"].wait_stream(torch.cuda.current_stream())
-    e0.record()
-    for ln in lanes:
-        ln["s"].wait_event(e0)
-    for i in range(e2e_steps):
-        e2e_step(i)
-    for ln in lanes:
-        torch.cuda.current_stream().wait_stream(ln["s"])
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_wall_ms = (time.perf_counter() - t_host0) * 1e3
-    for ln in lanes:
-        status = F.flowmm_last_device_status(ln["ws"])
-        if status != 0:
-            raise RuntimeError("device status (end to end): " + F.status_string(status))
-    e2e_ms = shard.max_over_ranks(e2e_ms, dev)
-    e2e_value = shard.aggregate_throughput(tokens_layers, world, e2e_ms / e2e_steps)
-    del lanes
+        for i in range(len(lanes)):
+            e2e_step(i)
+        barrier()
+        t_host0 = time.perf_counter()
+        for ln in lanes:
+            ln["s"].wait_stream(torch.cuda.current_stream())
+        e0.record()
+        for ln in lanes:
+            ln["s"].wait_event(e0)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        for ln in lanes:
+            torch.cuda.current_stream().wait_stream(ln["s"])
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        e2e_wall_ms = (time.perf_counter() - t_host0) * 1e3
+        for ln in lanes:
+            status = F.flowmm_last_device_status(ln["ws"])
+            if status != 0:
+                raise RuntimeError("device status (end to end): " + F.status_string(status))
+        e2e_ms = shard.max_over_ranks(e2e_ms, dev)
+        e2e_value = shard.aggregate_throughput(tokens_layers, world, e2e_ms / e2e_steps)
+        del lanes
+        return {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "wall_ms_per_step": round(e2e_wall_ms / e2e_steps, 4)}
+
+
+    try:
+        e2e = end_to_end()
+    except (RuntimeError, MemoryError) as exc:      # e.g. the host cannot pin a whole input set: say so, keep the line
+        if "device status" in str(exc):
+            raise
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+               "error": str(exc).splitlines()[0][:200]}
+    torch.cuda.synchronize()
 
     # the step this path feeds (not part of the timed metric): one decode query per head over every layer's
     # cache, full length against compressed; L2 flushed before every call, each call timed on its own
@@ -480,21 +580,22 @@ def run_ours(args):
                        "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "seq_len": wl.seq_len,
                        "window": wl.window, "budget_permille": args.permille, "n_keep": B,
                        "units_per_call": U, "match_pairs_fraction_of_dense": round(pairs / max(1.0, dense_pairs), 4),
-                       "launch": launch_mode,
+                       "launch": "plain flowmm_compress_layer calls",
                        "l2": "%d rotating input sets of %.0f MB (inputs larger than L2)" %
                        (n_sets, bytes_per_set / 1e6), "path": args.path, "parallelism": "units sharded, no collective"},
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps, "wall_ms_per_step": round(e2e_wall_ms / e2e_steps, 4)},
+            "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline,
             "kernels": {n: {k2: (round(v2, 5) if isinstance(v2, float) else v2) for k2, v2 in d.items()}
                         for n, d in kernels.items()},
         }
+        if graph_ms_step is not None:
+            line["graph_replay_ms_per_step"] = graph_ms_step
         if decode is not None:
             line["decode"] = decode
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(wl, args.permille, args.cpu_baseline_units)
+            line["cpu_baseline"] = cpu_baseline(wl, args.permille, args.cpu_baseline_units, args.cpu_seconds)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -23,7 +23,9 @@
  *     (size from flowmm_workspace_bytes, 256-byte aligned); its first word is a sticky
  *     device status, so the caller zero-fills the first 256 bytes once after allocating
  *     it.  Inputs are never written; outputs must not alias inputs.
- *   - n_units * n_kv_heads must not exceed 65535 per call (a CUDA grid dimension).
+ *   - n_units * n_kv_heads must not exceed 4 194 304 per call, and that product times the number of
+ *     128-token tiles of the context times the number of 128-row tiles of a KV head's proxy rows must
+ *     stay below 2^31 (work items are counted in 32 bits); else FLOWMM_ERR_SHAPE.
  *   - Q, K, V and the outputs have the element type `dtype`, head_dim contiguous, and the
  *     element strides given in the params (unit, head, token).  Base pointers must be
  *     16-byte aligned and every stride a multiple of 8 elements, else FLOWMM_ERR_ALIGN.
@@ -168,9 +170,16 @@ flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v,
  * flowmm_merge (same kernels, same fixed accumulation order, so the outputs are bit-identical).
  *
  * Limits and rules:
- *   - The scratch a problem needs is about 16 E + 28 (B + 1) + E / 4 bytes per (unit, KV head)
- *     plus (2 E / 64 + 2) * (8 head_dim + 16) bytes per (unit, KV head) of partial sums; if
- *     that exceeds the array the call returns FLOWMM_ERR_WORKSPACE and launches nothing.
+ *   - The scratch a problem needs, per (unit, KV head): 16 E + 16 (B + E / 64 + 1) + 12 (B + 1) + 4 B
+ *     bytes of slot lists, piece table and counters, 8 L bytes of per-token (slot, weight) pairs,
+ *     and (2 (E / 64) + 2) * (8 head_dim + 16) bytes of partial sums; every part is rounded up
+ *     to 256 bytes and 768 bytes are fixed.  If that exceeds the array the call returns
+ *     FLOWMM_ERR_WORKSPACE and launches nothing.
+ *   - A problem found on the device (a bounded wait that ran out) is recorded in a status word
+ *     inside the array, since there is no workspace to carry it: flowmm_merge_static_status
+ *     waits for the stream, returns that word (FLOWMM_OK or the first error recorded by any
+ *     call since the last read) and clears it.  Outputs of a call that reported an error are
+ *     not valid.
  *   - The first call on a device looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array and it keeps the previous call's contents;
@@ -181,6 +190,10 @@ flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v,
 flowmm_status flowmm_merge_static(const flowmm_params *p, const void *k, const void *v, const int32_t *retained_idx,
                                   const int32_t *evicted_idx, const int32_t *match, const float *match_sim,
                                   void *k_out, void *v_out, void *cuda_stream);
+flowmm_status flowmm_merge_static_status(void *cuda_stream);
+/* Test aid for the reader above: waits for the stream and stores `word` in the array's status word
+ * from the host, so that reading and clearing can be checked without making a kernel fail. */
+flowmm_status flowmm_merge_static_poke_status(int32_t word, void *cuda_stream);
 
 /*
  * Steps 1-5 in order on one stream: the whole per-layer FlowMM compression of Section 3.3.

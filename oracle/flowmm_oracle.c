@@ -10,8 +10,11 @@
  *
  * Inputs are float32 arrays holding the exact values the GPU receives (for
  * bf16 workloads: bf16 values widened to float32); all arithmetic is double.
- * OpenMP only spreads independent (unit, head) problems over cores; there is
- * no blocking, fusion or reordering inside a problem.
+ * OpenMP only spreads independent work over cores: (unit, head) problems, or,
+ * when a call has fewer of those than cores, the independent dot products of
+ * one attention row and the independent non-pivot rows of the matching step.
+ * Every value is computed by the same operations in the same order either way;
+ * there is no blocking, fusion or reordering inside a problem.
  *
  * Steps (notation: unit u, query head g, KV head h = g / G, window row a at
  * prompt position p_a = L - W + a, token i, modality m[i] in {0 text, 1 visual}):
@@ -94,8 +97,10 @@ int flowmm_oracle_score(const oracle_params *p, const float *q, const float *k, 
     if (Hkv <= 0 || Hq % Hkv != 0 || W < 1 || W > L) return 1;
     const int G = Hq / Hkv;
     const double scale = p->softmax_scale != 0.0 ? p->softmax_scale : 1.0 / sqrt((double)D);
+    /* few (unit, head) problems: the cores share the independent logits of one row instead */
+    const int by_head = U * Hkv >= flowmm_oracle_threads();
 
-#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+#pragma omp parallel for collapse(2) schedule(dynamic, 1) if (by_head)
     for (int u = 0; u < U; ++u) {
         for (int h = 0; h < Hkv; ++h) {
             const uint8_t *m = modality + (size_t)u * L;
@@ -109,10 +114,11 @@ int flowmm_oracle_score(const oracle_params *p, const float *q, const float *k, 
                     const int pa = L - W + a;               /* prompt position of this proxy token */
                     const float *qa = q + (((size_t)u * Hq + g) * W + a) * (size_t)D;
                     double mx = -INFINITY;
-                    for (int i = 0; i <= pa; ++i) {          /* causal: keys after p_a are masked */
+#pragma omp parallel for schedule(static) if (!by_head)
+                    for (int i = 0; i <= pa; ++i)            /* causal: keys after p_a are masked */
                         alpha[i] = scale * dotd(qa, kh + (size_t)i * D, D);
+                    for (int i = 0; i <= pa; ++i)
                         if (alpha[i] > mx) mx = alpha[i];
-                    }
                     double z = 0.0;
                     for (int i = 0; i <= pa; ++i) { alpha[i] = exp(alpha[i] - mx); z += alpha[i]; }
                     for (int i = 0; i <= pa; ++i) {
@@ -210,49 +216,50 @@ static double tau_effective(const oracle_params *p)
  * when the unit's strategy is intra-modal.  match = slot in [0,B) or -1,
  * sim = the winning similarity (0 when there is none), runner_up = the second
  * largest admissible similarity (-2 when there is none; used by tests to
- * measure how close a decision was).  row_step > 1 evaluates only every
- * row_step-th non-pivot and marks the others match = -2.
+ * measure how close a decision was).  row_select (optional, [U,Hkv,E] bytes)
+ * limits the work to the non-pivots whose byte is non-zero; the others are
+ * marked match = -2.
  */
 int flowmm_oracle_match(const oracle_params *p, const float *k, const double *importance, const uint8_t *modality,
                         const int32_t *retained, const int32_t *evicted, const int32_t *strategy,
-                        int32_t row_step, int32_t *match, double *sim, double *runner_up)
+                        const uint8_t *row_select, int32_t *match, double *sim, double *runner_up)
 {
     const int U = p->n_units, Hkv = p->n_kv_heads, D = p->head_dim, L = p->seq_len, B = p->n_keep;
     const int E = L - B;
     const double tau = tau_effective(p);
-    if (row_step < 1) row_step = 1;
-#pragma omp parallel for collapse(2) schedule(dynamic, 1)
-    for (int u = 0; u < U; ++u) {
-        for (int h = 0; h < Hkv; ++h) {
-            const uint8_t *m = modality + (size_t)u * L;
-            const float *kh = k + ((size_t)u * Hkv + h) * (size_t)L * D;
-            const double *imp = importance + ((size_t)u * Hkv + h) * (size_t)L;
-            const int32_t *r = retained + ((size_t)u * Hkv + h) * (size_t)B;
-            const int32_t *ev = evicted + ((size_t)u * Hkv + h) * (size_t)E;
-            const size_t base = ((size_t)u * Hkv + h) * (size_t)E;
-            for (int j = 0; j < E; ++j) {
-                if (j % row_step != 0) {
-                    match[base + j] = -2; sim[base + j] = 0.0;
-                    if (runner_up) runner_up[base + j] = -2.0;
-                    continue;
-                }
-                const int e = ev[j];
-                int best = -1;
-                double ubest = 0.0, usecond = -2.0;
-                for (int s = 0; s < B; ++s) {
-                    const int rs = r[s];
-                    if (!(imp[rs] <= tau)) continue;                       /* highly sensitive pivot: kept intact */
-                    if (strategy[u] == 0 && m[rs] != m[e]) continue;       /* intra-modal layer */
-                    const double us = flowmm_oracle_cosine(D, kh + (size_t)e * D, kh + (size_t)rs * D);
-                    if (best < 0) { best = s; ubest = us; }
-                    else if (us > ubest) { usecond = ubest; best = s; ubest = us; }   /* strict: ties keep lower slot */
-                    else if (us > usecond) usecond = us;
-                }
-                match[base + j] = best;
-                sim[base + j] = best >= 0 ? ubest : 0.0;
-                if (runner_up) runner_up[base + j] = usecond;
-            }
+    /* every non-pivot row of every (unit, head) is an independent problem */
+    const long long n_rows = (long long)U * Hkv * E;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (long long row = 0; row < n_rows; ++row) {
+        const int j = (int)(row % E);
+        const int h = (int)(row / E % Hkv);
+        const int u = (int)(row / E / Hkv);
+        const uint8_t *m = modality + (size_t)u * L;
+        const float *kh = k + ((size_t)u * Hkv + h) * (size_t)L * D;
+        const double *imp = importance + ((size_t)u * Hkv + h) * (size_t)L;
+        const int32_t *r = retained + ((size_t)u * Hkv + h) * (size_t)B;
+        const int32_t *ev = evicted + ((size_t)u * Hkv + h) * (size_t)E;
+        const size_t base = ((size_t)u * Hkv + h) * (size_t)E;
+        if (row_select && !row_select[base + j]) {
+            match[base + j] = -2; sim[base + j] = 0.0;
+            if (runner_up) runner_up[base + j] = -2.0;
+            continue;
         }
+        const int e = ev[j];
+        int best = -1;
+        double ubest = 0.0, usecond = -2.0;
+        for (int s = 0; s < B; ++s) {
+            const int rs = r[s];
+            if (!(imp[rs] <= tau)) continue;                       /* highly sensitive pivot: kept intact */
+            if (strategy[u] == 0 && m[rs] != m[e]) continue;       /* intra-modal layer */
+            const double us = flowmm_oracle_cosine(D, kh + (size_t)e * D, kh + (size_t)rs * D);
+            if (best < 0) { best = s; ubest = us; }
+            else if (us > ubest) { usecond = ubest; best = s; ubest = us; }   /* strict: ties keep lower slot */
+            else if (us > usecond) usecond = us;
+        }
+        match[base + j] = best;
+        sim[base + j] = best >= 0 ? ubest : 0.0;
+        if (runner_up) runner_up[base + j] = usecond;
     }
     return 0;
 }

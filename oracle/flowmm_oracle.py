@@ -138,8 +138,9 @@ def select(p: OracleParams, importance):
     return ret, evi
 
 
-def match(p: OracleParams, k, importance, modality, retained, evicted, strategy, row_step: int = 1):
-    """-> match [U,Hkv,E] int32, sim [U,Hkv,E], runner_up [U,Hkv,E] float64."""
+def match(p: OracleParams, k, importance, modality, retained, evicted, strategy, row_select=None):
+    """-> match [U,Hkv,E] int32, sim [U,Hkv,E], runner_up [U,Hkv,E] float64.  row_select (optional, bool
+    [U,Hkv,E]): only these non-pivots are evaluated, the others come back with match = -2."""
     k = _f32(k)
     imp = np.ascontiguousarray(importance, dtype=np.float64)
     m = np.ascontiguousarray(modality, dtype=np.uint8)
@@ -152,8 +153,12 @@ def match(p: OracleParams, k, importance, modality, retained, evicted, strategy,
     sim = np.zeros((p.n_units, p.n_kv_heads, E), dtype=np.float64)
     ru = np.zeros((p.n_units, p.n_kv_heads, E), dtype=np.float64)
     cp = p.c()
+    sel = None
+    if row_select is not None:
+        sel = np.ascontiguousarray(row_select, dtype=np.uint8)
+        assert sel.shape == mt.shape
     _load().flowmm_oracle_match(ctypes.byref(cp), _ptr(k), _ptr(imp), _ptr(m), _ptr(ret), _ptr(evi), _ptr(strat),
-                                ctypes.c_int32(row_step), _ptr(mt), _ptr(sim), _ptr(ru))
+                                _ptr(sel) if sel is not None else ctypes.c_void_p(0), _ptr(mt), _ptr(sim), _ptr(ru))
     return mt, sim, ru
 
 
@@ -175,7 +180,7 @@ def merge(p: OracleParams, k, v, retained, evicted, match_, sim):
 
 
 def compress_layer(p: OracleParams, q, k, v, modality, forced: Optional[Dict[str, np.ndarray]] = None,
-                   row_step: int = 1) -> Dict[str, np.ndarray]:
+                   row_select=None) -> Dict[str, np.ndarray]:
     """The whole path, step by step.  `forced` may replace the decision outputs of a
     step ("importance", "strategy", "retained"+"evicted", "match"+"match_sim") before
     the steps after it run; tests use it to follow a near-tie the other way."""
@@ -194,12 +199,12 @@ def compress_layer(p: OracleParams, q, k, v, modality, forced: Optional[Dict[str
     else:
         ret, evi = select(p, out["importance"])
     out["retained"], out["evicted"] = np.asarray(ret, dtype=np.int32), np.asarray(evi, dtype=np.int32)
-    mt, sim, ru = match(p, k, out["importance"], modality, out["retained"], out["evicted"], out["strategy"], row_step)
+    mt, sim, ru = match(p, k, out["importance"], modality, out["retained"], out["evicted"], out["strategy"], row_select)
     out["match_own"], out["match_sim_own"], out["runner_up"] = mt, sim, ru
     if "match" in forced:
         mt, sim = forced["match"], forced["match_sim"]
     out["match"], out["match_sim"] = np.asarray(mt, dtype=np.int32), np.asarray(sim, dtype=np.float64)
-    if row_step == 1:
+    if row_select is None:
         ko, vo, z = merge(p, k, v, out["retained"], out["evicted"], out["match"], out["match_sim"])
         out["k_out"], out["v_out"], out["weight_sum"] = ko, vo, z
     return out

@@ -31,6 +31,7 @@ EXPORTS = (
     "flowmm_profile_enable", "flowmm_profile_read", "flowmm_merge_static", "flowmm_selftest_wait_timeout",
     "flowmm_decode_workspace_bytes", "flowmm_decode_attention",
     "flowmm_full_flow_workspace_bytes", "flowmm_full_flow",
+    "flowmm_merge_static_status", "flowmm_merge_static_poke_status",
 )
 
 
@@ -121,6 +122,8 @@ def load() -> ctypes.CDLL:
         for name in EXPORTS[:8]:
             getattr(lib, name).restype = ctypes.c_int
         lib.flowmm_merge_static.restype = ctypes.c_int
+        lib.flowmm_merge_static_status.restype = ctypes.c_int
+        lib.flowmm_merge_static_poke_status.restype = ctypes.c_int
         lib.flowmm_selftest_wait_timeout.restype = ctypes.c_int
         lib.flowmm_decode_workspace_bytes.restype = ctypes.c_int
         lib.flowmm_decode_attention.restype = ctypes.c_int
@@ -224,6 +227,15 @@ def flowmm_merge_static(p: Params, k, v, retained_idx, evicted_idx, match, match
     cp = p.c(k=k, v=v, ko=k_out, vo=v_out)
     _check(load().flowmm_merge_static(ctypes.byref(cp), _p(k), _p(v), _p(retained_idx), _p(evicted_idx), _p(match),
                                       _p(match_sim), _p(k_out), _p(v_out), _stream()), "flowmm_merge_static")
+
+
+def flowmm_merge_static_status() -> int:
+    """Device status of the flowmm_merge_static calls since the last read (0 = ok); waits for the stream, clears."""
+    return int(load().flowmm_merge_static_status(_stream()))
+
+
+def flowmm_merge_static_poke_status(word: int):
+    _check(load().flowmm_merge_static_poke_status(ctypes.c_int32(word), _stream()), "flowmm_merge_static_poke_status")
 
 
 def flowmm_compress_layer(p: Params, q_win, k, v, modality, k_out, v_out, ws, importance=None, rho=None,

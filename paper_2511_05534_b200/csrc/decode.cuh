@@ -25,7 +25,7 @@ __device__ __forceinline__ float dec_ex2(float x) {
     return y;
 }
 
-// grid = (n_split, U*Hkv), block = 128.  GP = G rounded up to 1, 2, 4 or 8; D = head_dim.
+// grid = (U*Hkv, n_split), block = 128.  GP = G rounded up to 1, 2, 4 or 8; D = head_dim.
 // A group of D / kVec lanes shares a row (16 bytes per lane); the groups of a block take the keys of the
 // block's range in turn.  Dynamic shared memory: (rows groups per block) * GP * (D + 2) floats.
 template <typename T, int D, int GP>
@@ -33,8 +33,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
     constexpr int V = Elem<T>::kVec, LPR = D / V, GROUPS = kDecThreads / LPR;
     extern __shared__ float dec_smem[];                              // [GROUPS][GP][D + 2]
     const int tid = threadIdx.x, sub = tid % LPR, grp = tid / LPR;
-    const int uh = blockIdx.y, u = uh / A.Hkv, h = uh % A.Hkv;
-    const int lo = blockIdx.x * A.keys_per_split, hi = min(A.N, lo + A.keys_per_split);
+    const int uh = blockIdx.x, u = uh / A.Hkv, h = uh % A.Hkv;
+    const int lo = blockIdx.y * A.keys_per_split, hi = min(A.N, lo + A.keys_per_split);
     const T *kb = static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1] + sub * V;
     const T *vb = static_cast<const T *>(A.v) + u * A.vs[0] + h * A.vs[1] + sub * V;
     const T *qb = static_cast<const T *>(A.q) + ((int64_t)u * A.Hq + h * A.G) * D + sub * V;
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
             o = fmaf(rec[d], w, o);
             ls = fmaf(rec[D + 1], w, ls);
         }
-        float *dst = A.part + (((int64_t)uh * A.n_split + blockIdx.x) * A.G + g) * (D + 2);
+        float *dst = A.part + (((int64_t)uh * A.n_split + blockIdx.y) * A.G + g) * (D + 2);
         dst[d] = o;
         if (d == 0) { dst[D] = mx; dst[D + 1] = ls; }
     }

@@ -103,7 +103,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
     tc::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    const int uh = blockIdx.y, u = uh / A.Hkv, h = uh % A.Hkv, split = blockIdx.x;
+    const int uh = blockIdx.x, u = uh / A.Hkv, h = uh % A.Hkv, split = blockIdx.y;
     const int tiles_total = (A.N + kTile - 1) / kTile;
     const int t0 = split * A.tiles_per_split, nt = min(A.tiles_per_split, tiles_total - t0);
     const int key0 = t0 * kTile;

@@ -58,6 +58,10 @@ inline void profile_mark(const char *name, cudaStream_t st) {
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// (unit, head) pairs per call: they index grid.x of several launches and 32-bit item counters
+// (items = pairs x row tiles), so the bound is generous rather than a grid limit of 65535.
+constexpr int64_t kMaxHeadsPerCall = 1 << 22;
+
 // Where everything lives inside the caller's workspace.  One layout serves every entry point.
 struct Layout {
     size_t status, importance, cross_mass, rho, strategy, retained, evicted, match, match_sim;
@@ -166,7 +170,12 @@ flowmm_status validate(const flowmm_params *p) {
     if (p->n_q_heads % p->n_kv_heads != 0) return FLOWMM_ERR_SHAPE;
     if (p->head_dim != 64 && p->head_dim != 128) return FLOWMM_ERR_SHAPE;
     if (p->seq_len < 1 || p->window < 1 || p->window > p->seq_len) return FLOWMM_ERR_SHAPE;
-    if ((int64_t)p->n_units * p->n_kv_heads > 65535) return FLOWMM_ERR_SHAPE;
+    if ((int64_t)p->n_units * p->n_kv_heads > kMaxHeadsPerCall) return FLOWMM_ERR_SHAPE;
+    {   // work items (pairs x 128-row tiles of the context x 128-row tiles of a head's proxy rows) are counted in 32 bits
+        const int64_t tiles = (int64_t)p->n_units * p->n_kv_heads * ((p->seq_len + 127) / 128) *
+                              (((int64_t)p->n_q_heads / p->n_kv_heads * p->window + 127) / 128);
+        if (tiles > 0x7FFFFFFFll) return FLOWMM_ERR_SHAPE;
+    }
     if (p->n_keep < 1 || p->n_keep > p->seq_len) return FLOWMM_ERR_BUDGET;
     if (p->keep_window && p->n_keep < p->window) return FLOWMM_ERR_BUDGET;
     if (p->dtype != FLOWMM_F32 && p->dtype != FLOWMM_BF16) return FLOWMM_ERR_DTYPE;
@@ -318,7 +327,7 @@ flowmm_status run_score(const flowmm_params &p, const Layout &y, const void *q, 
     for (int i = 0; i < 3; ++i) { a.qs[i] = p.q_stride[i]; a.ks[i] = p.k_stride[i]; }
     const int GW = a.G * a.W;
     const int UH = p.n_units * p.n_kv_heads;
-    const dim3 g1(y.n_chunk1, (GW + kTile - 1) / kTile, UH), g2(y.n_chunk2, 1, UH);
+    const dim3 g1(UH, (GW + kTile - 1) / kTile, y.n_chunk1), g2(UH, y.n_chunk2);
     const size_t dyn = (size_t)3 * GW * sizeof(float);
     if (p.dtype == FLOWMM_BF16) {
         score_stats_simt<__nv_bfloat16><<<g1, kSimtThreads, 0, st>>>(a);
@@ -382,7 +391,7 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     match_prepare_kernel<<<UH, prep_threads, 0, st>>>(g);
     FLOWMM_LAUNCHED("match_prepare");
     if (!g.copy_here) {
-        match_gather_kernel<<<dim3((y.c_tot + 63) / 64, UH), 256, 0, st>>>(g);
+        match_gather_kernel<<<dim3(UH, (y.c_tot + 63) / 64), 256, 0, st>>>(g);
         FLOWMM_LAUNCHED("match_gather");
     }
 
@@ -457,7 +466,7 @@ flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, 
     a.Hkv = p.n_kv_heads; a.D = p.head_dim; a.L = p.seq_len; a.B = p.n_keep; a.E = E;
     a.tau_eff = tau_effective(p);
     for (int i = 0; i < 3; ++i) a.ks[i] = p.k_stride[i];
-    const dim3 grid((E + kTile - 1) / kTile, 1, p.n_units * p.n_kv_heads);
+    const dim3 grid(p.n_units * p.n_kv_heads, (E + kTile - 1) / kTile);
     if (p.dtype == FLOWMM_BF16) match_simt<__nv_bfloat16><<<grid, kSimtThreads, 0, st>>>(a);
     else match_simt<float><<<grid, kSimtThreads, 0, st>>>(a);
     FLOWMM_LAUNCHED("match_simt");
@@ -492,7 +501,7 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
         ma.tokmap = at<int2>(ws, y.tokmap); ma.L = p.seq_len; ma.B = p.n_keep; ma.E = E; ma.merge_mode = p.merge_mode;
         const int longest = E > p.n_keep ? E : p.n_keep;
         if (!map_ready) {
-            mtc::merge_map_kernel<<<dim3((longest + 255) / 256, UH), 256, 0, st>>>(ma);
+            mtc::merge_map_kernel<<<dim3(UH, (longest + 255) / 256), 256, 0, st>>>(ma);
             FLOWMM_LAUNCHED("merge_map");
         }
         CUtensorMap kmap, vmap;
@@ -844,7 +853,7 @@ extern "C" flowmm_status flowmm_full_flow(const flowmm_params *p, const void *q_
     uint32_t *bits = at<uint32_t>(ws, f.bits);
     const int mod_words = (p->seq_len + 31) / 32 + 8;                  // + slack: whole 256-key tiles are indexed
     if (use_tc(*p)) {
-        pack_modality_kernel<<<dim3((mod_words + 7) / 8, p->n_units), 256, 0, st>>>(modality, p->seq_len, mod_words, bits);
+        pack_modality_kernel<<<dim3(p->n_units, (mod_words + 7) / 8), 256, 0, st>>>(modality, p->seq_len, mod_words, bits);
         FLOWMM_LAUNCHED("pack_modality");
     }
     for (int t = 0; t < n_tiles; ++t) {
@@ -878,7 +887,7 @@ flowmm_status validate_decode(const flowmm_decode_params *p) {
     if (p->n_units < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_keys < 1) return FLOWMM_ERR_SHAPE;
     if (p->n_q_heads % p->n_kv_heads != 0 || p->n_q_heads / p->n_kv_heads > 8) return FLOWMM_ERR_SHAPE;
     if (p->head_dim != 64 && p->head_dim != 128) return FLOWMM_ERR_SHAPE;
-    if ((int64_t)p->n_units * p->n_kv_heads > 65535) return FLOWMM_ERR_SHAPE;
+    if ((int64_t)p->n_units * p->n_kv_heads > kMaxHeadsPerCall) return FLOWMM_ERR_SHAPE;
     if (p->dtype != FLOWMM_F32 && p->dtype != FLOWMM_BF16) return FLOWMM_ERR_DTYPE;
     if (!(p->softmax_scale >= 0.f)) return FLOWMM_ERR_SHAPE;
     if (p->path != FLOWMM_PATH_AUTO && p->path != FLOWMM_PATH_SIMT) return FLOWMM_ERR_SHAPE;
@@ -929,7 +938,7 @@ DecodePlan decode_plan(const flowmm_decode_params &p) {
 template <typename T, int D>
 flowmm_status launch_decode(const DecodeArgs &a, int uh, int n_q, cudaStream_t st) {
     constexpr int groups = kDecThreads / (D / Elem<T>::kVec);
-    const dim3 grid(a.n_split, uh);
+    const dim3 grid(uh, a.n_split);
     const int gp = a.G <= 1 ? 1 : a.G <= 2 ? 2 : a.G <= 4 ? 4 : 8;
     const size_t smem = (size_t)groups * gp * (D + 2) * sizeof(float);
     switch (gp) {
@@ -952,21 +961,18 @@ flowmm_status launch_decode_tc(const flowmm_decode_params &p, const DecodeArgs &
     const uint32_t box[4] = {64, dtc::kTile, 1, 1};
     if (!tc::make_bf16_map(&kmap, a.k, 4, dims, ks, box) || !tc::make_bf16_map(&vmap, a.v, 4, dims, vs, box))
         return FLOWMM_ERR_CUDA;
-    static bool configured = false;      // per process; the attribute is the same on every device
-    if (!configured) {
-        if (cudaFuncSetAttribute(dtc::decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)dtc::kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(dtc::decode_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess)
-            return FLOWMM_ERR_CUDA;
-        configured = true;
-    }
+    // (function attributes belong to the current device: set on every call, like the other launchers)
+    if (cudaFuncSetAttribute(dtc::decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)dtc::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(dtc::decode_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        return FLOWMM_ERR_CUDA;
     dtc::Args t;
     t.q = static_cast<const __nv_bfloat16 *>(a.q); t.part = a.part; t.out = a.out; t.status = status;
     t.tickets = status + 64;
     t.Hq = a.Hq; t.Hkv = a.Hkv; t.G = a.G; t.N = a.N; t.n_split = a.n_split; t.tiles_per_split = a.keys_per_split;
     t.scale_log2 = a.scale_log2;
-    dtc::decode_tc_kernel<<<dim3(a.n_split, uh), dtc::kThreads, dtc::kSmemBytes, st>>>(kmap, vmap, t);
+    dtc::decode_tc_kernel<<<dim3(uh, a.n_split), dtc::kThreads, dtc::kSmemBytes, st>>>(kmap, vmap, t);
     FLOWMM_LAUNCHED("decode_tc");
     return FLOWMM_OK;
 }
@@ -1062,11 +1068,13 @@ flowmm_status merge_static_base(void **base) {
     return FLOWMM_OK;
 }
 
-// The part of the workspace layout that the merge step touches, packed from offset 0.
+// The part of the workspace layout that the merge step touches, packed behind the array's status word
+// (the first 256 bytes, where flowmm_merge_static_status finds it whatever the problem's shape).
 Layout make_merge_layout(const flowmm_params &p) {
     Layout y = {};
-    size_t o = 0;
+    size_t o = 256;
     layout_merge(y, p, [&](size_t bytes) { const size_t at = o; o += align256(bytes); return at; });
+    y.merge_status = 0;
     y.total = o;
     return y;
 }
@@ -1091,9 +1099,27 @@ extern "C" flowmm_status flowmm_merge_static(const flowmm_params *p, const void 
     FLOWMM_TRY(check_device());
     void *base = nullptr;
     FLOWMM_TRY(merge_static_base(&base));
-    // Nothing in this scratch has to start at zero: the CSR arrays are written in full before they
-    // are read and a partial-sum record is only read for pieces that wrote it in the same call.
+    // Nothing in this scratch has to start at zero: the slot lists, the piece table, the work counter and
+    // the arrival counters are written (or cleared) by this call's first kernel before they are read, a
+    // partial-sum record is only read for pieces that wrote it in the same call, and the status word is
+    // sticky on purpose (the loader zero-fills the array; flowmm_merge_static_status clears the word).
     return run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, base,
                      static_cast<cudaStream_t>(cuda_stream));
 }
 
+extern "C" flowmm_status flowmm_merge_static_status(void *cuda_stream) {
+    FLOWMM_TRY(check_device());
+    void *base = nullptr;
+    FLOWMM_TRY(merge_static_base(&base));
+    return flowmm_last_device_status(base, cuda_stream);
+}
+
+// Test hook of the reader above: stores `word` in the array's status word from the host, in stream order.
+extern "C" flowmm_status flowmm_merge_static_poke_status(int32_t word, void *cuda_stream) {
+    FLOWMM_TRY(check_device());
+    void *base = nullptr;
+    FLOWMM_TRY(merge_static_base(&base));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(base, &word, sizeof(word), cudaMemcpyHostToDevice, st) != cudaSuccess) return FLOWMM_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? FLOWMM_OK : FLOWMM_ERR_CUDA;
+}

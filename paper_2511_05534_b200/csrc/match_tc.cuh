@@ -122,10 +122,10 @@ __global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs
 }
 
 // The gather step of the preparation as a kernel of its own for long candidate lists, so that many
-// CTAs share a head's rows.  grid = (ceil(Ctot / 64), U*Hkv), block = 256.
+// CTAs share a head's rows.  grid = (U*Hkv, ceil(Ctot / 64)), block = 256.
 __global__ void __launch_bounds__(256) match_gather_kernel(const MatchPrepArgs A) {
-    const int lo = blockIdx.x * 64;
-    match_gather_rows(A, blockIdx.y, lo, min(A.Ctot, lo + 64), threadIdx.x, blockDim.x);
+    const int lo = blockIdx.y * 64;
+    match_gather_rows(A, blockIdx.x, lo, min(A.Ctot, lo + 64), threadIdx.x, blockDim.x);
 }
 
 struct MatchTcArgs {

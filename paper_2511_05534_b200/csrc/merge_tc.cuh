@@ -65,9 +65,9 @@ struct MapArgs {
     int L, B, E, merge_mode;
 };
 
-// grid = (ceil(max(E, B) / 256), UH)
+// grid = (UH, ceil(max(E, B) / 256))
 __global__ void __launch_bounds__(256) merge_map_kernel(const MapArgs A) {
-    const int uh = blockIdx.y, i = blockIdx.x * 256 + threadIdx.x;
+    const int uh = blockIdx.x, i = blockIdx.y * 256 + threadIdx.x;
     int2 *map = A.tokmap + (int64_t)uh * A.L;
     if (i < A.E) {
         const int tok = A.evicted[(int64_t)uh * A.E + i];

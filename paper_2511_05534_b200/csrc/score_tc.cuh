@@ -213,7 +213,7 @@ __global__ void flow_combine_kernel(const float2 *row_part, const float *row_cro
 
 // Packs the modality map: word w of a unit holds keys 32 w .. 32 w + 31 (bit set = visual; keys past the prompt: 0).
 __global__ void pack_modality_kernel(const uint8_t *modality, int L, int n_words, uint32_t *bits) {
-    const int u = blockIdx.y, w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int u = blockIdx.x, w = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (w >= n_words) return;
     const int key = 32 * w + lane;
     const uint32_t word = __ballot_sync(0xFFFFFFFFu, key < L && modality[(int64_t)u * L + key] != 0);

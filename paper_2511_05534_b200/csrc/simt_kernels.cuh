@@ -79,15 +79,15 @@ struct ScoreArgs {
 };
 
 // Pass 1 of Eq. 8: per proxy row the running maximum and exp-sum of its causal logits over one
-// chunk of keys.  grid = (n_chunk1, row tiles of G*W, U*Hkv).
+// chunk of keys.  grid = (U*Hkv, row tiles of G*W, n_chunk1).
 template <typename T>
 __global__ void __launch_bounds__(kSimtThreads) score_stats_simt(const ScoreArgs A) {
     __shared__ SimtTiles sm;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-    const int uh = blockIdx.z, u = uh / A.Hkv, h = uh % A.Hkv;
+    const int uh = blockIdx.x, u = uh / A.Hkv, h = uh % A.Hkv;
     const int GW = A.G * A.W;
     const int row0 = blockIdx.y * kTile;
-    const int key_lo = blockIdx.x * A.chunk1, key_hi = min(A.L, key_lo + A.chunk1);
+    const int key_lo = blockIdx.z * A.chunk1, key_hi = min(A.L, key_lo + A.chunk1);
     const T *q = static_cast<const T *>(A.q) + u * A.qs[0];
     const T *k = static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
 
@@ -141,13 +141,13 @@ __global__ void __launch_bounds__(kSimtThreads) score_stats_simt(const ScoreArgs
         }
         const int r = row0 + ty * 4 + i;
         if (tx == 0 && r < GW)
-            A.row_part[((int64_t)uh * GW + r) * A.n_chunk1 + blockIdx.x] = make_float2(m[i], l[i]);
+            A.row_part[((int64_t)uh * GW + r) * A.n_chunk1 + blockIdx.z] = make_float2(m[i], l[i]);
     }
 }
 
 // Pass 2 of Eq. 8 and the modality split of Eq. 7: logits are recomputed, normalised with the
 // row statistics of pass 1, summed down the columns into the importance, and summed per head
-// over the keys of the other modality.  grid = (n_chunk2, 1, U*Hkv); dynamic shared memory:
+// over the keys of the other modality.  grid = (U*Hkv, n_chunk2); dynamic shared memory:
 // 3*G*W floats.
 template <typename T>
 __global__ void __launch_bounds__(kSimtThreads) score_colsum_simt(const ScoreArgs A) {
@@ -157,8 +157,8 @@ __global__ void __launch_bounds__(kSimtThreads) score_colsum_simt(const ScoreArg
     const int GW = A.G * A.W;
     float *row_max = dyn, *row_inv = dyn + GW, *row_cross = dyn + 2 * GW;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-    const int uh = blockIdx.z, u = uh / A.Hkv, h = uh % A.Hkv;
-    const int key_lo = blockIdx.x * A.chunk2, key_hi = min(A.L, key_lo + A.chunk2);
+    const int uh = blockIdx.x, u = uh / A.Hkv, h = uh % A.Hkv;
+    const int key_lo = blockIdx.y * A.chunk2, key_hi = min(A.L, key_lo + A.chunk2);
     const T *q = static_cast<const T *>(A.q) + u * A.qs[0];
     const T *k = static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
     const uint8_t *mod = A.modality + (int64_t)u * A.L;
@@ -234,7 +234,7 @@ __global__ void __launch_bounds__(kSimtThreads) score_colsum_simt(const ScoreArg
     for (int g = tid; g < A.G; g += kSimtThreads) {
         float s = 0.f;
         for (int a = 0; a < A.W; ++a) s += row_cross[g * A.W + a];
-        A.cross_part[((int64_t)u * A.Hq + h * A.G + g) * A.n_chunk2 + blockIdx.x] = s;
+        A.cross_part[((int64_t)u * A.Hq + h * A.G + g) * A.n_chunk2 + blockIdx.y] = s;
     }
 }
 
@@ -315,12 +315,12 @@ struct MatchArgs {
 };
 
 // Eq. 9 and Eq. 10: cosine similarity of 64 non-pivots against every pivot, gated argmax per row.
-// grid = (ceil(E / 64), 1, U*Hkv).
+// grid = (U*Hkv, ceil(E / 64)).
 template <typename T>
 __global__ void __launch_bounds__(kSimtThreads) match_simt(const MatchArgs A) {
     __shared__ SimtTiles sm;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-    const int uh = blockIdx.z, u = uh / A.Hkv, h = uh % A.Hkv;
+    const int uh = blockIdx.x, u = uh / A.Hkv, h = uh % A.Hkv;
     const T *k = static_cast<const T *>(A.k) + u * A.ks[0] + h * A.ks[1];
     const int *ret = A.retained + (int64_t)uh * A.B;
     const int *evi = A.evicted + (int64_t)uh * A.E;
@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(kSimtThreads) match_simt(const MatchArgs A) {
     const float *rn = A.rn + (int64_t)uh * A.L;
     const uint8_t *mod = A.modality + (int64_t)u * A.L;
     const bool intra = A.strategy[u] == 0;
-    const int j0 = blockIdx.x * kTile;
+    const int j0 = blockIdx.y * kTile;
 
     float rne[4], best[4];
     int bests[4];

@@ -40,14 +40,16 @@ inline bool make_bf16_map(CUtensorMap *map, const void *base, int rank, const ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// SM count of the current device (a benign race: every thread would store the same value).
 inline int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    }
-    return n;
+    constexpr int kSlots = 64;
+    static int n[kSlots] = {};
+    int dev = 0, count = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < kSlots && n[dev] != 0) return n[dev];
+    cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev);
+    if (dev >= 0 && dev < kSlots) n[dev] = count;
+    return count;
 }
 
 }  // namespace tc

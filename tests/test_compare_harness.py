@@ -57,3 +57,33 @@ def test_rejects_planted_mistakes(mistake):
         g["retained"][0, 0, :2] = g["retained"][0, 0, :2][::-1]
     with pytest.raises(C.ParityError):
         C.compare(p, d["q"], d["k"], d["v"], d["modality"], g, bf16_out=False)
+
+
+def test_sampled_rows_judge_only_what_the_oracle_matched():
+    """With a row sample the harness still rejects a wrong match inside the sample, and a slot that received a
+    non-pivot outside the sample is left out of the K/V comparison instead of being judged on the other side's
+    own match."""
+    p, d, g = _case()
+    E = p.seq_len - p.n_keep
+    sel = np.random.default_rng(3).random((1, p.n_kv_heads, E)) < 0.5     # the sample compare() draws for seed 3
+    stats = C.compare(p, d["q"], d["k"], d["v"], d["modality"], g, bf16_out=False, row_fraction=0.5, row_seed=3)
+    assert stats["match_rows_checked"] == int(sel.sum()) < stats["match_rows_total"]
+    assert stats["kv_rows_checked"] < stats["kv_rows_total"]
+    # a wrong match outside the sample, with K/V that follow it: not judged (and not accepted as checked either)
+    h = 2
+    outside = [j for j in np.nonzero(~sel[0, h])[0] if g["match"][0, h, j] >= 0]
+    inside = [j for j in np.nonzero(sel[0, h])[0] if g["match"][0, h, j] >= 0]
+    bad = {key: val.copy() for key, val in g.items()}
+    j = outside[0]
+    bad["match"][0, h, j] = (bad["match"][0, h, j] + 1) % p.n_keep
+    forced = O.merge(p, d["k"], d["v"], bad["retained"], bad["evicted"], bad["match"], bad["match_sim"])
+    bad["k_out"], bad["v_out"] = forced[0], forced[1]
+    C.compare(p, d["q"], d["k"], d["v"], d["modality"], bad, bf16_out=False, row_fraction=0.5, row_seed=3)
+    with pytest.raises(C.ParityError):                                     # the full check does see it
+        C.compare(p, d["q"], d["k"], d["v"], d["modality"], bad, bf16_out=False)
+    # the same mistake inside the sample is rejected
+    bad = {key: val.copy() for key, val in g.items()}
+    j = inside[0]
+    bad["match"][0, h, j] = (bad["match"][0, h, j] + 1) % p.n_keep
+    with pytest.raises(C.ParityError):
+        C.compare(p, d["q"], d["k"], d["v"], d["modality"], bad, bf16_out=False, row_fraction=0.5, row_seed=3)
