@@ -202,12 +202,36 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 }
                 ok = ok && tc::mbar_wait(bar(kBarAccFull + team), (i >> 2) & 1, abort_flag, A.status);
                 tc::tc_fence_after();
-                float best = -INFINITY;
-                int best_cc = -1;
+                // Running winner among the columns walked so far; candidates are laid out text group first, each group by
+                // ascending slot, so the first maximum of a group is its lowest slot.  A token of a cross-modal layer sees
+                // both groups: the text group's winner is set aside at the first visual block and the two meet by
+                // (similarity, slot), so that equal similarities go to the lower slot.
+                float best = -INFINITY, val_a = -INFINITY;
+                int best_cc = -1, slot_a = -1;
+                auto resolve = [&]() -> int {                        // slot of the running winner: lowest column of its group that holds the maximum
+                    if (best_cc < 0) return -1;
+                    int idx = 0;
+#pragma unroll
+                    for (int q4 = 1; q4 >= 0; --q4) {
+                        const float4 w = tc::lds128(wrow + q4 * 16);
+                        if (w.w == best) idx = 4 * q4 + 3;
+                        if (w.z == best) idx = 4 * q4 + 2;
+                        if (w.y == best) idx = 4 * q4 + 1;
+                        if (w.x == best) idx = 4 * q4;
+                    }
+                    return __float_as_int(tc::lds32(md + slot_off + (best_cc + idx) * 4));
+                };
+                const int park_blk = intra ? -1 : (t0 >> 4);
                 for (int blk = 0; blk < nb_all; ++blk) {
                     uint32_t acc[16];
                     tc::tmem_ld16(trow + blk * 16, acc);
                     tc::tmem_ld_wait(acc);
+                    if (blk == park_blk) {
+                        slot_a = resolve();
+                        val_a = best;
+                        best = -INFINITY;
+                        best_cc = -1;
+                    }
                     if (blk >= blo && blk < bhi) {
                         float v[16];
 #pragma unroll
@@ -235,19 +259,8 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 tc::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(bar(kBarSetFree + team));   // this warp has read the accumulator
-                int slot = -1;
-                if (best_cc >= 0) {
-                    int idx = 0;
-#pragma unroll
-                    for (int q4 = 1; q4 >= 0; --q4) {                // lowest column that holds the maximum
-                        const float4 w = tc::lds128(wrow + q4 * 16);
-                        if (w.w == best) idx = 4 * q4 + 3;
-                        if (w.z == best) idx = 4 * q4 + 2;
-                        if (w.y == best) idx = 4 * q4 + 1;
-                        if (w.x == best) idx = 4 * q4;
-                    }
-                    slot = __float_as_int(tc::lds32(md + slot_off + (best_cc + idx) * 4));
-                }
+                int slot = resolve();
+                if (match_better(val_a, slot_a, best, slot)) { best = val_a; slot = slot_a; }
                 if (in_range && my_rank >= 0 && ok) {                // a non-pivot: report its match
                     float sim = 0.f;
                     if (slot >= 0 && ssq > 0.f) sim = best * rsqrtf(ssq);

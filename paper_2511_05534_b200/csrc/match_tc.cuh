@@ -192,6 +192,89 @@ __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) 
     return match_plan<S>(A, item, match_raw(A, item));
 }
 
+// The inner step of the epilogue, written out in PTX so that it stays at the instruction count the tensor core
+// leaves room for (a 128 x 256 accumulator is refilled in 1024 clocks; four warps per scheduler share its columns).
+// One block of 16 accumulator columns of this thread's row: similarities = accumulators x the candidates' reciprocal
+// norms (packed pairs); each of the block's two groups of 8 columns gives a maximum; a group that beats the row's
+// running maximum - strictly, so that the earlier column keeps a tie, and never with NaN (= no candidate there) -
+// becomes the winner: its 8 values go to the row's stash in shared memory (predicated stores, no branch) and `tag`
+// records which group it was (kTag, kTag + 8: its column offset inside the warp's share of the tile).
+//   taddr   TMEM address of the block for this warp's lanes        scales   shared address of the block's 16 norms
+//   stash   shared address of the row's 8-float stash
+#define FLOWMM_MB_MUL(i, j, k) "mov.b64 t" #k ", {a" #i ", a" #j "};\n\tmul.rn.f32x2 t" #k ", t" #k ", s" #k ";\n\tmov.b64 {v" #i ", v" #j "}, t" #k ";\n\t"
+template <int kTag>
+__device__ __forceinline__ void match_block16(uint32_t taddr, uint32_t scales, uint32_t stash, float &best, int &tag) {
+    asm volatile(
+        "{\n\t"
+        ".reg .b32 a<16>;\n\t"
+        ".reg .b64 s<8>, t<8>;\n\t"
+        ".reg .f32 v<16>, m<6>, q<2>;\n\t"
+        ".reg .pred p<2>;\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {a0, a1, a2, a3, a4, a5, a6, a7, a8, a9, a10, a11, a12, a13, a14, a15}, [%2];\n\t"
+        "ld.shared.v2.b64 {s0, s1}, [%3];\n\t"
+        "ld.shared.v2.b64 {s2, s3}, [%3 + 16];\n\t"
+        "ld.shared.v2.b64 {s4, s5}, [%3 + 32];\n\t"
+        "ld.shared.v2.b64 {s6, s7}, [%3 + 48];\n\t"
+        "tcgen05.wait::ld.sync.aligned;\n\t"
+        FLOWMM_MB_MUL(0, 1, 0) FLOWMM_MB_MUL(2, 3, 1) FLOWMM_MB_MUL(4, 5, 2) FLOWMM_MB_MUL(6, 7, 3)
+        FLOWMM_MB_MUL(8, 9, 4) FLOWMM_MB_MUL(10, 11, 5) FLOWMM_MB_MUL(12, 13, 6) FLOWMM_MB_MUL(14, 15, 7)
+        "max.f32 m0, v0, v1, v2;\n\t"
+        "max.f32 m1, v3, v4, v5;\n\t"
+        "max.f32 m2, v6, v7;\n\t"
+        "max.f32 m3, v8, v9, v10;\n\t"
+        "max.f32 m4, v11, v12, v13;\n\t"
+        "max.f32 m5, v14, v15;\n\t"
+        "max.f32 q0, m0, m1, m2;\n\t"
+        "max.f32 q1, m3, m4, m5;\n\t"
+        "setp.gt.f32 p0, q0, %0;\n\t"
+        "@p0 st.shared.v4.f32 [%4], {v0, v1, v2, v3};\n\t"
+        "@p0 st.shared.v4.f32 [%4 + 16], {v4, v5, v6, v7};\n\t"
+        "@p0 mov.f32 %0, q0;\n\t"
+        "@p0 mov.s32 %1, %5;\n\t"
+        "setp.gt.f32 p1, q1, %0;\n\t"
+        "@p1 st.shared.v4.f32 [%4], {v8, v9, v10, v11};\n\t"
+        "@p1 st.shared.v4.f32 [%4 + 16], {v12, v13, v14, v15};\n\t"
+        "@p1 mov.f32 %0, q1;\n\t"
+        "@p1 mov.s32 %1, %6;\n\t"
+        "}"
+        : "+f"(best), "+r"(tag)
+        : "r"(taddr), "r"(scales), "r"(stash), "n"(kTag), "n"(kTag + 8)
+        : "memory");
+}
+#undef FLOWMM_MB_MUL
+
+// kN blocks in a row, starting at block 0 of the warp's share.
+template <int kN, int kI = 0>
+__device__ __forceinline__ void match_blocks(uint32_t taddr, uint32_t scales, uint32_t stash, float &best, int &tag) {
+    if constexpr (kI < kN) {
+        match_block16<16 * kI>(taddr + 16 * kI, scales + 64 * kI, stash, best, tag);
+        match_blocks<kN, kI + 1>(taddr, scales, stash, best, tag);
+    }
+}
+
+// Of two (similarity, slot) results the larger similarity wins and equal similarities go to the lower slot
+// (slot < 0: no result).
+__device__ __forceinline__ bool match_better(float va, int sa, float vb, int sb) {
+    return sa >= 0 && (sb < 0 || va > vb || (va == vb && sa < sb));
+}
+
+// Squared norm of 64 bf16 elements of a key row in an operand stage (one 128-byte swizzled row: 16-byte units
+// XOR-ed with the row index), as packed pairs.
+__device__ __forceinline__ float row_half_ssq(uint32_t row_addr, int row) {
+    float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int un = 0; un < 8; ++un) {
+        const float4 rawf = tc::lds128(row_addr + ((un ^ (row & 7)) << 4));
+        const uint32_t w[4] = {__float_as_uint(rawf.x), __float_as_uint(rawf.y), __float_as_uint(rawf.z), __float_as_uint(rawf.w)};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {            // a bf16 is the upper half of the fp32 with the same value
+            const float2 x = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+            acc = tc::ffma2(x, x, acc);
+        }
+    }
+    return acc.x + acc.y;
+}
+
 // Persistent kernel, one CTA per SM; item = (unit, head, tile of 256 tokens).
 template <class S>
 __global__ void __launch_bounds__(tcs::kThreads, 1)
@@ -199,7 +282,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 const MatchTcArgs A) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr int kMtCols = S::kCols;
-    const typename S::Ctx c = S::setup(smem_raw, &k_map, &cand_map, A.status, 4);
+    constexpr int kPer = kMtCols / 32;                           // blocks of 16 columns a warp takes of a full tile
+    const typename S::Ctx c = S::setup(smem_raw, &k_map, &cand_map, A.status, 8);
     if (!c.ok) return;
     auto plan = [&](int item) { return match_plan<S>(A, item).tp; };
     if (c.warp == 0) {
@@ -208,8 +292,10 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         if (c.lane == 0) S::mma_issuer(c, A.n_items, plan, A.status);
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
+        const int b0 = kPer * c.colhalf;                         // first block of this warp's share of a tile
         const uint32_t wrow = c.epi_addr() + row * 32;          // 8 floats per row
         const uint32_t prow = c.partner_addr() + row * 32;      // the other column half's
+        const uint32_t t_lane = c.tmem_base + c.group * kMtCols + b0 * 16 + ((uint32_t)(c.quarter * 32) << 16);
         int k = 0, bt = 0, n_mine = 0;
         bool ok = true;
         // what an item needs from global memory is fetched one item ahead: its plan values, the token's
@@ -236,30 +322,46 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             const int token = p.rt * kMtItemRows + c.group * kMtRows + row;
             const bool in_range = token < A.L;
             const bool row_masked = p.intra && p.mixed;
-            float best = -INFINITY;
-            int best_cc = -1;
-            float ssq = 0.f;                                         // squared norm of this row's key
+            const int *slots = A.cand_slot + (int64_t)p.uh * A.Ctot;
+            // Running winner of this row among the warp's columns: its similarity (still times the row's norm), the tile
+            // it came from and the group of 8 columns inside the warp's share of that tile; the group's values are in
+            // the stash.  Candidates are laid out text group first, each group by ascending slot, so within a group the
+            // first maximum is the lowest slot; where a row sees both groups (a cross-modal layer) the text group's
+            // winner is set aside when the first visual column comes up, and the two meet by (similarity, slot).
+            float best = -INFINITY, before = -INFINITY;
+            int tag = -1, best_tile = 0;
+            float val_a = -INFINITY;                                 // the winner set aside
+            int slot_a = -1;
+            bool parked = p.intra;                                   // (an intra-modal row sees one group only)
+            float ssq = 0.f;                                         // squared norm of this row's key, this warp's half of it
+            // slot of the running winner: the lowest column of its group that holds the maximum
+            auto resolve = [&]() -> int {
+                if (tag < 0) return -1;
+                int idx = 0;
+#pragma unroll
+                for (int q4 = 1; q4 >= 0; --q4) {
+                    const float4 w = tc::lds128(wrow + q4 * 16);
+                    if (w.w == best) idx = 4 * q4 + 3;
+                    if (w.z == best) idx = 4 * q4 + 2;
+                    if (w.y == best) idx = 4 * q4 + 1;
+                    if (w.x == best) idx = 4 * q4;
+                }
+                return slots[p.lo + best_tile * kMtCols + b0 * 16 + tag + idx];
+            };
+            auto park = [&](int t) {
+                if (best > before) best_tile = t;                   // the winner may be of this tile's earlier blocks
+                slot_a = resolve();
+                val_a = best;
+                best = -INFINITY; before = -INFINITY; tag = -1;
+                parked = true;
+            };
             if (!active) {
                 if (!p.tp.empty()) bt += p.tp.n_tiles;               // keep the B-tile count in step
             } else {
-                if (c.colhalf == 0) {
-                    // the token's key row sits in this half's A stage (128-byte rows, 16-byte units XOR-swizzled by
-                    // the row index): read it once for the norm while the first MMAs run, then hand the stage back
+                {   // the token's key row sits in this half's A stage: each of the row's two warps reads one 64-element
+                    // half of it for the norm while the first MMAs run, then hands the stage back
                     ok = S::a_wait(c, n_mine, A.status);
-                    const uint32_t a_half = c.a_addr(n_mine) + row * 128;
-#pragma unroll
-                    for (int kh = 0; kh < 2; ++kh) {
-#pragma unroll
-                        for (int un = 0; un < 8; ++un) {
-                            const float4 rawf = tc::lds128(a_half + kh * (tcs::kAHalf / 2) + ((un ^ (row & 7)) << 4));
-                            const uint4 raw = make_uint4(__float_as_uint(rawf.x), __float_as_uint(rawf.y), __float_as_uint(rawf.z),
-                                                         __float_as_uint(rawf.w));
-                            float x[8];
-                            Elem<__nv_bfloat16>::unpack(raw, x);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) ssq = fmaf(x[e], x[e], ssq);
-                        }
-                    }
+                    ssq = row_half_ssq(c.a_addr(n_mine) + c.colhalf * (tcs::kAHalf / 2) + row * 128, row);
                     S::a_release(c, n_mine++);
                 }
                 for (int t = 0; ok && t < p.tp.n_tiles; ++t, ++k, ++bt) {
@@ -268,22 +370,21 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     ok = S::extra_wait(c, bt, A.status) && S::acc_wait(c, k, A.status);
                     if (!ok) break;
                     const uint32_t scale4 = c.extra(bt);             // reciprocal norms of this tile's candidates
-                    // one block of 16 columns; kMasked: rows of the tile differ in which columns they may take
-                    auto block = [&](auto masked_tag, int blk, uint32_t (&acc)[16]) {
-                        constexpr bool kMasked = decltype(masked_tag)::value;
-                        const int cc = col0 + blk * 16;
-                        float v[16];
+                    const int n_blocks = (ncols + 15) >> 4;
+                    if (row_masked) {
+                        // intra-modal layer, tile with tokens of both modalities: rows differ in which columns they may take
+                        S::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) {
+                            const int cc = col0 + blk * 16;
+                            float v[16];
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {     // a column that is no candidate has scale NaN and never wins
-                            const float4 s4 = tc::lds128(scale4 + (blk * 4 + q4) * 16);
-                            v[4 * q4 + 0] = __uint_as_float(acc[4 * q4 + 0]) * s4.x;
-                            v[4 * q4 + 1] = __uint_as_float(acc[4 * q4 + 1]) * s4.y;
-                            v[4 * q4 + 2] = __uint_as_float(acc[4 * q4 + 2]) * s4.z;
-                            v[4 * q4 + 3] = __uint_as_float(acc[4 * q4 + 3]) * s4.w;
-                        }
-                        if constexpr (kMasked) {             // intra-modal layer, tile with tokens of both modalities
-                            // admissible columns of this row
-                            int r1hi = p.n_text, r2lo = p.t0, r2hi = p.t0 + p.n_vis;
+                            for (int q4 = 0; q4 < 4; ++q4) {     // a column that is no candidate has scale NaN and never wins
+                                const float4 s4 = tc::lds128(scale4 + (blk * 4 + q4) * 16);
+                                v[4 * q4 + 0] = __uint_as_float(acc[4 * q4 + 0]) * s4.x;
+                                v[4 * q4 + 1] = __uint_as_float(acc[4 * q4 + 1]) * s4.y;
+                                v[4 * q4 + 2] = __uint_as_float(acc[4 * q4 + 2]) * s4.z;
+                                v[4 * q4 + 3] = __uint_as_float(acc[4 * q4 + 3]) * s4.w;
+                            }
+                            int r1hi = p.n_text, r2lo = p.t0, r2hi = p.t0 + p.n_vis;   // admissible columns of this row
                             if (my_mod == 0) r2hi = r2lo; else r1hi = 0;
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
@@ -291,26 +392,48 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                                 const bool valid = (col < r1hi) || (col >= r2lo && col < r2hi);
                                 v[j] = valid ? v[j] : -INFINITY;
                             }
-                        }
 #pragma unroll
-                        for (int g = 0; g < 2; ++g) {        // two groups of 8 columns, in column order
-                            const float q8 = tc::max3(tc::max3(v[8 * g], v[8 * g + 1], v[8 * g + 2]),
-                                                      tc::max3(v[8 * g + 3], v[8 * g + 4], v[8 * g + 5]),
-                                                      fmaxf(v[8 * g + 6], v[8 * g + 7]));
-                            if (q8 > best) {                 // strict: an earlier group keeps a tie (false for NaN)
-                                best = q8;
-                                best_cc = cc + 8 * g;
-                                // keep the 8 columns to find the exact one later
-                                tc::sts128(wrow, v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3]);
-                                tc::sts128(wrow + 16, v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]);
+                            for (int g = 0; g < 2; ++g) {        // two groups of 8 columns, in column order
+                                const float q8 = tc::max3(tc::max3(v[8 * g], v[8 * g + 1], v[8 * g + 2]),
+                                                          tc::max3(v[8 * g + 3], v[8 * g + 4], v[8 * g + 5]),
+                                                          fmaxf(v[8 * g + 6], v[8 * g + 7]));
+                                if (q8 > best) {                 // strict: an earlier group keeps a tie (false for NaN)
+                                    best = q8;
+                                    tag = (blk - b0) * 16 + 8 * g;
+                                    best_tile = t;
+                                    tc::sts128(wrow, v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3]);
+                                    tc::sts128(wrow + 16, v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]);
+                                }
+                            }
+                        });
+                    } else {
+                        const int nb = min(n_blocks - b0, kPer);     // blocks of this warp in this tile (may be <= 0)
+                        // block before which the text group's winner is set aside (>= nb: not in this tile)
+                        const int pk = parked ? kPer : max(0, (p.t0 - (col0 + b0 * 16)) >> 4);
+                        const uint32_t sc = scale4 + b0 * 64;
+                        before = best;
+                        if (nb == kPer && pk >= kPer) {
+                            match_blocks<kPer>(t_lane, sc, wrow, best, tag);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < kPer; ++i) {
+                                if (i < nb) {
+                                    if (i == pk) park(t);
+                                    switch (i) {                     // (the block's tag is a compile-time constant)
+                                        case 0: match_block16<0>(t_lane, sc, wrow, best, tag); break;
+                                        case 1: match_block16<16>(t_lane + 16, sc + 64, wrow, best, tag); break;
+                                        case 2: match_block16<32>(t_lane + 32, sc + 128, wrow, best, tag); break;
+                                        case 3: match_block16<48>(t_lane + 48, sc + 192, wrow, best, tag); break;
+                                        case 4: match_block16<64>(t_lane + 64, sc + 256, wrow, best, tag); break;
+                                        case 5: match_block16<80>(t_lane + 80, sc + 320, wrow, best, tag); break;
+                                        case 6: match_block16<96>(t_lane + 96, sc + 384, wrow, best, tag); break;
+                                        default: match_block16<112>(t_lane + 112, sc + 448, wrow, best, tag); break;
+                                    }
+                                }
                             }
                         }
-                    };
-                    const int n_blocks = (ncols + 15) >> 4;
-                    if (row_masked)
-                        S::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::true_type{}, blk, acc); });
-                    else
-                        S::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) { block(std::false_type{}, blk, acc); });
+                        if (best > before) best_tile = t;            // the winner moved into this tile
+                    }
                     S::acc_release(c);
                 }
             }
@@ -319,24 +442,17 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             // ends for both right after them)
             // this warp's result for the row: similarity (still times the row's norm) and pivot slot
             int slot = -1;
-            if (best_cc >= 0 && ok) {
-                int idx = 0;
-#pragma unroll
-                for (int q4 = 1; q4 >= 0; --q4) {                    // lowest column that holds the maximum
-                    const float4 w = tc::lds128(wrow + q4 * 16);
-                    if (w.w == best) idx = 4 * q4 + 3;
-                    if (w.z == best) idx = 4 * q4 + 2;
-                    if (w.y == best) idx = 4 * q4 + 1;
-                    if (w.x == best) idx = 4 * q4;
-                }
-                slot = A.cand_slot[(int64_t)p.uh * A.Ctot + best_cc + idx];
+            if (ok && active) {
+                slot = resolve();
+                if (match_better(val_a, slot_a, best, slot)) { best = val_a; slot = slot_a; }
             }
-            // the upper column half hands its result to the lower one, which owns the row's output
-            if (c.colhalf == 1) tc::sts128(wrow, best, __int_as_float(slot), 0.f, 0.f);
+            // the upper column half hands its result and its half of the norm to the lower one, which owns the row's output
+            if (c.colhalf == 1) tc::sts128(wrow, best, __int_as_float(slot), ssq, 0.f);
             ok = !S::pair_meet(c, !ok);                            // (both warps of a row go on, or neither)
             if (c.colhalf == 0 && ok) {
                 const float4 other = tc::lds128(prow);
-                if (other.x > best) { best = other.x; slot = __float_as_int(other.y); }    // a tie stays with the lower columns
+                if (match_better(other.x, __float_as_int(other.y), best, slot)) { best = other.x; slot = __float_as_int(other.y); }
+                ssq += other.z;
                 if (in_range) {
                     const int j = my_rank;
                     if (j >= 0) {                                    // a non-pivot: report its match
