@@ -192,63 +192,97 @@ __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) 
     return match_plan<S>(A, item, match_raw(A, item));
 }
 
-// The inner step of the epilogue, written out in PTX so that it stays at the instruction count the tensor core
-// leaves room for (a 128 x 256 accumulator is refilled in 1024 clocks; four warps per scheduler share its columns).
+// The inner step of the epilogue, written out in PTX so that it stays inside what the tensor core leaves room for:
+// a 128 x 256 accumulator is refilled in 1024 clocks, in which the four schedulers issue 4096 warp instructions for its
+// 1024 warp-wide elements, and the tensor core's operand reads already take three quarters of the shared-memory
+// bandwidth, so the epilogue must not stage anything through shared memory.
 // One block of 16 accumulator columns of this thread's row: similarities = accumulators x the candidates' reciprocal
-// norms (packed pairs); each of the block's two groups of 8 columns gives a maximum; a group that beats the row's
-// running maximum - strictly, so that the earlier column keeps a tie, and never with NaN (= no candidate there) -
-// becomes the winner: its 8 values go to the row's stash in shared memory (predicated stores, no branch) and `tag`
-// records which group it was (kTag, kTag + 8: its column offset inside the warp's share of the tile).
+// norms (packed pairs; the norms are the block's only shared-memory reads); each similarity then carries its column in
+// its four lowest mantissa bits (15 - column, so that of equal similarities the lower column is the larger number; the
+// change is below 2^-19 relative, far inside the margin the decision is judged with); one maximum over the 16 tagged
+// values; the block's maximum with the tag cleared is compared with the row's running maximum `best`: a block that
+// beats it - strictly, so that an earlier block keeps a tie, and never with NaN (= no candidate there) - replaces it
+// and `win` records where it was: 16 x block number + tag.
 //   taddr   TMEM address of the block for this warp's lanes        scales   shared address of the block's 16 norms
-//   stash   shared address of the row's 8-float stash
-#define FLOWMM_MB_MUL(i, j, k) "mov.b64 t" #k ", {a" #i ", a" #j "};\n\tmul.rn.f32x2 t" #k ", t" #k ", s" #k ";\n\tmov.b64 {v" #i ", v" #j "}, t" #k ";\n\t"
-template <int kTag>
-__device__ __forceinline__ void match_block16(uint32_t taddr, uint32_t scales, uint32_t stash, float &best, int &tag) {
-    asm volatile(
-        "{\n\t"
-        ".reg .b32 a<16>;\n\t"
-        ".reg .b64 s<8>, t<8>;\n\t"
-        ".reg .f32 v<16>, m<6>, q<2>;\n\t"
-        ".reg .pred p<2>;\n\t"
+// (TMEM is read 32 columns at a time: a read has a cost of its own that does not shrink with its width, and sixteen
+// warps reading 16 columns each time kept the tensor core waiting for its accumulators.)
+#define FLOWMM_MB_MUL2(i, j, k, ti, tj)                                                                        \
+    "mov.b64 t0, {a" #i ", a" #j "};\n\tmul.rn.f32x2 t0, t0, s" #k ";\n\tmov.b64 {a" #i ", a" #j "}, t0;\n\t"    \
+    "lop3.b32 a" #i ", a" #i ", 0xFFFFFFF0, " #ti ", 0xEA;\n\t"                                                \
+    "lop3.b32 a" #j ", a" #j ", 0xFFFFFFF0, " #tj ", 0xEA;\n\t"
+#define FLOWMM_MB_LDS(OFF)                                     \
+    "ld.shared.v2.b64 {s0, s1}, [%3 + " #OFF "];\n\t"          \
+    "ld.shared.v2.b64 {s2, s3}, [%3 + " #OFF " + 16];\n\t"     \
+    "ld.shared.v2.b64 {s4, s5}, [%3 + " #OFF " + 32];\n\t"     \
+    "ld.shared.v2.b64 {s6, s7}, [%3 + " #OFF " + 48];\n\t"
+// 16 columns held in registers a<c0> .. a<c15>: products, tags, maximum, comparison with the running maximum;
+// WIN = 16 x block number, as an asm operand reference
+#define FLOWMM_MB_STEP(c0, c1, c2, c3, c4, c5, c6, c7, c8, c9, c10, c11, c12, c13, c14, c15, WIN)               \
+    FLOWMM_MB_MUL2(c0, c1, 0, 15, 14) FLOWMM_MB_MUL2(c2, c3, 1, 13, 12) FLOWMM_MB_MUL2(c4, c5, 2, 11, 10)       \
+    FLOWMM_MB_MUL2(c6, c7, 3, 9, 8) FLOWMM_MB_MUL2(c8, c9, 4, 7, 6) FLOWMM_MB_MUL2(c10, c11, 5, 5, 4)           \
+    FLOWMM_MB_MUL2(c12, c13, 6, 3, 2) FLOWMM_MB_MUL2(c14, c15, 7, 1, 0)                                         \
+    "max.f32 m0, a" #c0 ", a" #c1 ", a" #c2 ";\n\t"                                                             \
+    "max.f32 m1, a" #c3 ", a" #c4 ", a" #c5 ";\n\t"                                                             \
+    "max.f32 m2, a" #c6 ", a" #c7 ", a" #c8 ";\n\t"                                                             \
+    "max.f32 m3, a" #c9 ", a" #c10 ", a" #c11 ";\n\t"                                                           \
+    "max.f32 m4, a" #c12 ", a" #c13 ", a" #c14 ";\n\t"                                                          \
+    "max.f32 m0, m0, m1, m2;\n\t"                                                                               \
+    "max.f32 m3, m3, m4, a" #c15 ";\n\t"                                                                        \
+    "max.f32 q0, m0, m3;\n\t"                                                                                   \
+    "and.b32 qm, q0, 0xFFFFFFF0;\n\t"                                                                           \
+    "setp.gt.f32 p0, qm, %0;\n\t"                                                                               \
+    "@p0 mov.b32 %0, qm;\n\t"                                                                                   \
+    "@p0 lop3.b32 %1, q0, 15, " WIN ", 0xEA;\n\t"
+#define FLOWMM_MB_HEAD                 \
+    "{\n\t"                            \
+    ".reg .b32 a<32>, qm;\n\t"         \
+    ".reg .b64 s<8>, t0;\n\t"          \
+    ".reg .f32 m<5>, q0;\n\t"          \
+    ".reg .pred p0;\n\t"
+
+// Block number kBlk (16 columns) of the warp's share of the tile.
+template <int kBlk>
+__device__ __forceinline__ void match_block16(uint32_t taddr, uint32_t scales, float &best, int &win) {
+    asm volatile(FLOWMM_MB_HEAD
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {a0, a1, a2, a3, a4, a5, a6, a7, a8, a9, a10, a11, a12, a13, a14, a15}, [%2];\n\t"
-        "ld.shared.v2.b64 {s0, s1}, [%3];\n\t"
-        "ld.shared.v2.b64 {s2, s3}, [%3 + 16];\n\t"
-        "ld.shared.v2.b64 {s4, s5}, [%3 + 32];\n\t"
-        "ld.shared.v2.b64 {s6, s7}, [%3 + 48];\n\t"
+        FLOWMM_MB_LDS(0)
         "tcgen05.wait::ld.sync.aligned;\n\t"
-        FLOWMM_MB_MUL(0, 1, 0) FLOWMM_MB_MUL(2, 3, 1) FLOWMM_MB_MUL(4, 5, 2) FLOWMM_MB_MUL(6, 7, 3)
-        FLOWMM_MB_MUL(8, 9, 4) FLOWMM_MB_MUL(10, 11, 5) FLOWMM_MB_MUL(12, 13, 6) FLOWMM_MB_MUL(14, 15, 7)
-        "max.f32 m0, v0, v1, v2;\n\t"
-        "max.f32 m1, v3, v4, v5;\n\t"
-        "max.f32 m2, v6, v7;\n\t"
-        "max.f32 m3, v8, v9, v10;\n\t"
-        "max.f32 m4, v11, v12, v13;\n\t"
-        "max.f32 m5, v14, v15;\n\t"
-        "max.f32 q0, m0, m1, m2;\n\t"
-        "max.f32 q1, m3, m4, m5;\n\t"
-        "setp.gt.f32 p0, q0, %0;\n\t"
-        "@p0 st.shared.v4.f32 [%4], {v0, v1, v2, v3};\n\t"
-        "@p0 st.shared.v4.f32 [%4 + 16], {v4, v5, v6, v7};\n\t"
-        "@p0 mov.f32 %0, q0;\n\t"
-        "@p0 mov.s32 %1, %5;\n\t"
-        "setp.gt.f32 p1, q1, %0;\n\t"
-        "@p1 st.shared.v4.f32 [%4], {v8, v9, v10, v11};\n\t"
-        "@p1 st.shared.v4.f32 [%4 + 16], {v12, v13, v14, v15};\n\t"
-        "@p1 mov.f32 %0, q1;\n\t"
-        "@p1 mov.s32 %1, %6;\n\t"
+        FLOWMM_MB_STEP(0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, "%4")
         "}"
-        : "+f"(best), "+r"(tag)
-        : "r"(taddr), "r"(scales), "r"(stash), "n"(kTag), "n"(kTag + 8)
+        : "+f"(best), "+r"(win)
+        : "r"(taddr), "r"(scales), "n"(16 * kBlk)
         : "memory");
 }
-#undef FLOWMM_MB_MUL
 
-// kN blocks in a row, starting at block 0 of the warp's share.
+// Blocks kBlk and kBlk + 1 (32 columns) with one TMEM read.
+template <int kBlk>
+__device__ __forceinline__ void match_block32(uint32_t taddr, uint32_t scales, float &best, int &win) {
+    asm volatile(FLOWMM_MB_HEAD
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {a0, a1, a2, a3, a4, a5, a6, a7, a8, a9, a10, a11, a12, a13, a14, a15, "
+        "a16, a17, a18, a19, a20, a21, a22, a23, a24, a25, a26, a27, a28, a29, a30, a31}, [%2];\n\t"
+        FLOWMM_MB_LDS(0)
+        "tcgen05.wait::ld.sync.aligned;\n\t"
+        FLOWMM_MB_STEP(0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, "%4")
+        FLOWMM_MB_LDS(64)
+        FLOWMM_MB_STEP(16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, "%5")
+        "}"
+        : "+f"(best), "+r"(win)
+        : "r"(taddr), "r"(scales), "n"(16 * kBlk), "n"(16 * kBlk + 16)
+        : "memory");
+}
+#undef FLOWMM_MB_MUL2
+#undef FLOWMM_MB_LDS
+#undef FLOWMM_MB_STEP
+#undef FLOWMM_MB_HEAD
+
+// Blocks kI .. kN - 1 of the warp's share, two at a time.
 template <int kN, int kI = 0>
-__device__ __forceinline__ void match_blocks(uint32_t taddr, uint32_t scales, uint32_t stash, float &best, int &tag) {
-    if constexpr (kI < kN) {
-        match_block16<16 * kI>(taddr + 16 * kI, scales + 64 * kI, stash, best, tag);
-        match_blocks<kN, kI + 1>(taddr, scales, stash, best, tag);
+__device__ __forceinline__ void match_blocks(uint32_t taddr, uint32_t scales, float &best, int &win) {
+    if constexpr (kI + 1 < kN) {
+        match_block32<kI>(taddr + 16 * kI, scales + 64 * kI, best, win);
+        match_blocks<kN, kI + 2>(taddr, scales, best, win);
+    } else if constexpr (kI < kN) {
+        match_block16<kI>(taddr + 16 * kI, scales + 64 * kI, best, win);
     }
 }
 
@@ -293,8 +327,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     } else {
         const int lane = c.lane, row = c.quarter * 32 + lane;
         const int b0 = kPer * c.colhalf;                         // first block of this warp's share of a tile
-        const uint32_t wrow = c.epi_addr() + row * 32;          // 8 floats per row
-        const uint32_t prow = c.partner_addr() + row * 32;      // the other column half's
+        const uint32_t wrow = c.epi_addr() + row * 16;          // hand-over slot of this row
+        const uint32_t prow = c.partner_addr() + row * 16;      // the other column half's
         const uint32_t t_lane = c.tmem_base + c.group * kMtCols + b0 * 16 + ((uint32_t)(c.quarter * 32) << 16);
         int k = 0, bt = 0, n_mine = 0;
         bool ok = true;
@@ -323,36 +357,27 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             const bool in_range = token < A.L;
             const bool row_masked = p.intra && p.mixed;
             const int *slots = A.cand_slot + (int64_t)p.uh * A.Ctot;
-            // Running winner of this row among the warp's columns: its similarity (still times the row's norm), the tile
-            // it came from and the group of 8 columns inside the warp's share of that tile; the group's values are in
-            // the stash.  Candidates are laid out text group first, each group by ascending slot, so within a group the
-            // first maximum is the lowest slot; where a row sees both groups (a cross-modal layer) the text group's
-            // winner is set aside when the first visual column comes up, and the two meet by (similarity, slot).
+            // Running winner of this row among the warp's columns: its similarity (still times the row's norm, four
+            // lowest mantissa bits cleared), the tile it came from, and in `win` the block of 16 columns inside the warp's
+            // share of that tile (x 16) with 15 - column inside the block.  Candidates are laid out text group first, each group by ascending
+            // slot, so within a group the first maximum is the lowest slot; where a row sees both groups (a cross-modal
+            // layer) the text group's winner is set aside when the first visual column comes up, and the two meet by
+            // (similarity, slot).
             float best = -INFINITY, before = -INFINITY;
-            int tag = -1, best_tile = 0;
+            int win = -1, best_tile = 0;
             float val_a = -INFINITY;                                 // the winner set aside
             int slot_a = -1;
             bool parked = p.intra;                                   // (an intra-modal row sees one group only)
             float ssq = 0.f;                                         // squared norm of this row's key, this warp's half of it
-            // slot of the running winner: the lowest column of its group that holds the maximum
-            auto resolve = [&]() -> int {
-                if (tag < 0) return -1;
-                int idx = 0;
-#pragma unroll
-                for (int q4 = 1; q4 >= 0; --q4) {
-                    const float4 w = tc::lds128(wrow + q4 * 16);
-                    if (w.w == best) idx = 4 * q4 + 3;
-                    if (w.z == best) idx = 4 * q4 + 2;
-                    if (w.y == best) idx = 4 * q4 + 1;
-                    if (w.x == best) idx = 4 * q4;
-                }
-                return slots[p.lo + best_tile * kMtCols + b0 * 16 + tag + idx];
+            auto resolve = [&]() -> int {                            // slot of the running winner
+                if (win < 0) return -1;
+                return slots[p.lo + best_tile * kMtCols + (b0 + (win >> 4)) * 16 + 15 - (win & 15)];
             };
             auto park = [&](int t) {
                 if (best > before) best_tile = t;                   // the winner may be of this tile's earlier blocks
                 slot_a = resolve();
                 val_a = best;
-                best = -INFINITY; before = -INFINITY; tag = -1;
+                best = -INFINITY; before = -INFINITY; win = -1;
                 parked = true;
             };
             if (!active) {
@@ -373,12 +398,12 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     const int n_blocks = (ncols + 15) >> 4;
                     if (row_masked) {
                         // intra-modal layer, tile with tokens of both modalities: rows differ in which columns they may take
-                        S::for_each_block16(c, n_blocks, [&](int blk, uint32_t (&acc)[16]) {
-                            const int cc = col0 + blk * 16;
+                        S::for_each_block16(c, n_blocks, [&](int bl, uint32_t (&acc)[16]) {
+                            const int cc = col0 + bl * 16;
                             float v[16];
 #pragma unroll
                             for (int q4 = 0; q4 < 4; ++q4) {     // a column that is no candidate has scale NaN and never wins
-                                const float4 s4 = tc::lds128(scale4 + (blk * 4 + q4) * 16);
+                                const float4 s4 = tc::lds128(scale4 + (bl * 4 + q4) * 16);
                                 v[4 * q4 + 0] = __uint_as_float(acc[4 * q4 + 0]) * s4.x;
                                 v[4 * q4 + 1] = __uint_as_float(acc[4 * q4 + 1]) * s4.y;
                                 v[4 * q4 + 2] = __uint_as_float(acc[4 * q4 + 2]) * s4.z;
@@ -386,24 +411,19 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                             }
                             int r1hi = p.n_text, r2lo = p.t0, r2hi = p.t0 + p.n_vis;   // admissible columns of this row
                             if (my_mod == 0) r2hi = r2lo; else r1hi = 0;
+                            float q = -INFINITY;
+                            int qj = 0;
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
+                            for (int j = 0; j < 16; ++j) {           // columns in ascending order; NaN never wins
                                 const int col = cc + j;
                                 const bool valid = (col < r1hi) || (col >= r2lo && col < r2hi);
-                                v[j] = valid ? v[j] : -INFINITY;
+                                const float x = __uint_as_float(__float_as_uint(v[j]) & 0xFFFFFFF0u);   // as the unmasked path rounds it
+                                if (valid && x > q) { q = x; qj = j; }
                             }
-#pragma unroll
-                            for (int g = 0; g < 2; ++g) {        // two groups of 8 columns, in column order
-                                const float q8 = tc::max3(tc::max3(v[8 * g], v[8 * g + 1], v[8 * g + 2]),
-                                                          tc::max3(v[8 * g + 3], v[8 * g + 4], v[8 * g + 5]),
-                                                          fmaxf(v[8 * g + 6], v[8 * g + 7]));
-                                if (q8 > best) {                 // strict: an earlier group keeps a tie (false for NaN)
-                                    best = q8;
-                                    tag = (blk - b0) * 16 + 8 * g;
-                                    best_tile = t;
-                                    tc::sts128(wrow, v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3]);
-                                    tc::sts128(wrow + 16, v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]);
-                                }
+                            if (q > best) {                          // strict: an earlier block keeps a tie
+                                best = q;
+                                win = (bl - b0) * 16 + 15 - qj;
+                                best_tile = t;
                             }
                         });
                     } else {
@@ -413,21 +433,19 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                         const uint32_t sc = scale4 + b0 * 64;
                         before = best;
                         if (nb == kPer && pk >= kPer) {
-                            match_blocks<kPer>(t_lane, sc, wrow, best, tag);
+                            match_blocks<kPer>(t_lane, sc, best, win);
                         } else {
+                            // (the group boundary is a multiple of 32 columns, the warp's share starts at one: pairs of blocks)
 #pragma unroll
-                            for (int i = 0; i < kPer; ++i) {
+                            for (int i = 0; i < kPer; i += 2) {
                                 if (i < nb) {
                                     if (i == pk) park(t);
-                                    switch (i) {                     // (the block's tag is a compile-time constant)
-                                        case 0: match_block16<0>(t_lane, sc, wrow, best, tag); break;
-                                        case 1: match_block16<16>(t_lane + 16, sc + 64, wrow, best, tag); break;
-                                        case 2: match_block16<32>(t_lane + 32, sc + 128, wrow, best, tag); break;
-                                        case 3: match_block16<48>(t_lane + 48, sc + 192, wrow, best, tag); break;
-                                        case 4: match_block16<64>(t_lane + 64, sc + 256, wrow, best, tag); break;
-                                        case 5: match_block16<80>(t_lane + 80, sc + 320, wrow, best, tag); break;
-                                        case 6: match_block16<96>(t_lane + 96, sc + 384, wrow, best, tag); break;
-                                        default: match_block16<112>(t_lane + 112, sc + 448, wrow, best, tag); break;
+                                    const bool two = i + 1 < nb;
+                                    switch (i) {                     // (the block's number is a compile-time constant)
+                                        case 0: if (two) match_block32<0>(t_lane, sc, best, win); else match_block16<0>(t_lane, sc, best, win); break;
+                                        case 2: if (two) match_block32<2>(t_lane + 32, sc + 128, best, win); else match_block16<2>(t_lane + 32, sc + 128, best, win); break;
+                                        case 4: if (two) match_block32<4>(t_lane + 64, sc + 256, best, win); else match_block16<4>(t_lane + 64, sc + 256, best, win); break;
+                                        default: if (two) match_block32<6>(t_lane + 96, sc + 384, best, win); else match_block16<6>(t_lane + 96, sc + 384, best, win); break;
                                     }
                                 }
                             }
