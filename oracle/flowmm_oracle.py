@@ -223,3 +223,46 @@ def decode_attention(q, k, v, scale: float = 0.0) -> np.ndarray:
     if rc != 0:
         raise ValueError("oracle decode_attention: bad shape (code %d)" % rc)
     return out
+
+
+def recompress(p: OracleParams, q_win, k_cache, v_cache, row_modality) -> Dict[str, np.ndarray]:
+    """Re-compression of a cache that has grown during decoding (Eq. 3 appends one row per step; the paper runs
+    the compression of Section 3.3 once, after prefill, and does not say what happens afterwards).
+
+    The reading taken: the current cache of a KV head - the rows an earlier compression left, in order, followed by
+    the rows appended since - is treated as that head's context of length L' = p.seq_len, and the steps of
+    Section 3.3 run on it again with the proxy window taken from the W most recent queries (q_win):
+      * a row that came out of an earlier merge is an ordinary token now; its modality is that of the pivot it
+        was merged into, which is why modality is given per head and row (row_modality [U, Hkv, L']): after a
+        compression the heads of a layer no longer hold the same tokens;
+      * importance is taken afresh from the current window (nothing is carried over), the causal mask follows
+        the row order (window row a sees cache rows 0 .. L' - W + a), which is the true mask whenever at least W
+        rows have been appended;
+      * rho stays a property of the layer: the mean over all query heads of the layer (Eq. 6), each head's
+        cross-modal mass measured against its own KV head's row modalities; one strategy per unit;
+      * merge weights are those of Eq. 5's reading again (a row's earlier merges are not counted).
+    Returns the step outputs shaped per (unit, KV head), `row_modality_out` [U, Hkv, B'] for the next round,
+    rho [U] and strategy [U].
+    """
+    U, Hq, Hkv, D, L, W, B = p.n_units, p.n_q_heads, p.n_kv_heads, p.head_dim, p.seq_len, p.window, p.n_keep
+    G = Hq // Hkv
+    q, k, v = _f32(q_win), _f32(k_cache), _f32(v_cache)
+    m = np.ascontiguousarray(row_modality, dtype=np.uint8)
+    assert q.shape == (U, Hq, W, D) and k.shape == (U, Hkv, L, D) and v.shape == k.shape and m.shape == (U, Hkv, L)
+    # every (unit, KV head) as a problem of its own with one KV head, its G query heads and its own modality map
+    ph = OracleParams(U * Hkv, G, 1, D, L, W, B, p.softmax_scale, p.theta, p.tau, p.tau_mode, p.flow_mode,
+                      p.merge_mode, p.keep_window)
+    qh, kh, vh, mh = q.reshape(U * Hkv, G, W, D), k.reshape(U * Hkv, 1, L, D), v.reshape(U * Hkv, 1, L, D), m.reshape(U * Hkv, L)
+    imp, cross, total = score(ph, qh, kh, mh)
+    # Eq. 6 over all query heads of the layer
+    rho, strat = layer_flow(p, cross.reshape(U, Hq), total.reshape(U, Hq))
+    ret, evi = select(ph, imp)
+    mt, sim, _ = match(ph, kh, imp, mh, ret, evi, np.repeat(strat, Hkv))
+    ko, vo, _ = merge(ph, kh, vh, ret, evi, mt, sim)
+    E = L - B
+    return {
+        "importance": imp.reshape(U, Hkv, L), "cross": cross.reshape(U, Hq), "rho": rho, "strategy": strat,
+        "retained": ret.reshape(U, Hkv, B), "evicted": evi.reshape(U, Hkv, E), "match": mt.reshape(U, Hkv, E),
+        "match_sim": sim.reshape(U, Hkv, E), "k_out": ko.reshape(U, Hkv, B, D), "v_out": vo.reshape(U, Hkv, B, D),
+        "row_modality_out": np.take_along_axis(mh, ret.reshape(U * Hkv, B).astype(np.int64), -1).reshape(U, Hkv, B),
+    }
