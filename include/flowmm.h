@@ -57,7 +57,8 @@ typedef enum {
     FLOWMM_ERR_ALIGN = 6,
     FLOWMM_ERR_CUDA = 7,               /* a CUDA runtime call or launch failed */
     FLOWMM_ERR_TIMEOUT = 8,            /* device status: a bounded wait inside a kernel ran out */
-    FLOWMM_ERR_UNSUPPORTED_DEVICE = 9
+    FLOWMM_ERR_UNSUPPORTED_DEVICE = 9,
+    FLOWMM_ERR_INDEX = 10              /* debug build only: an index list or a computed index was out of range */
 } flowmm_status;
 
 typedef enum { FLOWMM_F32 = 0, FLOWMM_BF16 = 1 } flowmm_dtype;
@@ -208,6 +209,33 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
                                     void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Re-compression of a cache that has grown during decoding.  Eq. 3 appends one key / value row per decoded token;
+ * the paper runs the compression of Section 3.3 once, after prefill, and does not say what follows.  The reading
+ * offered here: the current cache of a KV head - the rows an earlier compression left, in order, then the rows
+ * appended since - is treated as that head's context of L = seq_len rows, and steps 1-5 run on it again with the
+ * proxy window taken from the W most recent queries.  A row that came out of an earlier merge is an ordinary token
+ * with the modality of the pivot it was merged into; after a compression the heads of a layer no longer hold the
+ * same tokens, so modality is given per head and row.  Importance is taken afresh from the window (the causal mask
+ * follows the row order, exact once at least W rows have been appended); rho is still the layer's, the mean over
+ * all query heads (Eq. 6), each head measured against its own rows; merge weights as in flowmm_merge.
+ *   q_win            [U, Hq, W, D]   queries of the W most recent positions
+ *   k_cache, v_cache [U, Hkv, L, D]  the cache rows, strides p->k_stride / p->v_stride
+ *   row_modality     [U, Hkv, L] uint8
+ *   k_out, v_out     [U, Hkv, B, D]; row_modality_out [U, Hkv, B] uint8 (the kept rows' modalities, for the next round)
+ *   importance ... match_sim: optional diagnostics (may be NULL), shaped as in flowmm_compress_layer but per
+ *   KV head throughout; rho, strategy [U].
+ * The unit stride of q, k, v and the outputs must equal heads x head stride (dense over heads), else
+ * FLOWMM_ERR_ALIGN.  Scratch: flowmm_recompress_workspace_bytes.  B == L returns the cache unchanged (the plain
+ * append of Eq. 3).
+ */
+flowmm_status flowmm_recompress_workspace_bytes(const flowmm_params *p, size_t *bytes);
+flowmm_status flowmm_recompress(const flowmm_params *p, const void *q_win, const void *k_cache, const void *v_cache,
+                                const uint8_t *row_modality, void *k_out, void *v_out, uint8_t *row_modality_out,
+                                float *importance, float *rho, int32_t *strategy, int32_t *retained_idx,
+                                int32_t *evicted_idx, int32_t *match, float *match_sim,
+                                void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * The step before the compression path: the cross-modal interaction ratio of Eq. 6 and Eq. 7 taken
  * literally, over every query row of the prefill (both the text-to-visual and the visual-to-text
  * term), instead of over the proxy window that flowmm_score uses.  Causal softmax attention of all
@@ -268,6 +296,16 @@ flowmm_status flowmm_selftest_wait_timeout(void *ws, void *cuda_stream);
 
 /* Number of kernels the most recent compute entry point of this thread enqueued. */
 int32_t flowmm_last_launch_count(void);
+
+/*
+ * 1 if the library was compiled with -DFLOWMM_DEBUG, else 0.  The debug build stands in for a memory checker:
+ * flowmm_match, flowmm_merge and flowmm_merge_static first check the index lists they are given (inside
+ * [0, L), strictly ascending; matches inside [-1, B)), wait for that check and return FLOWMM_ERR_INDEX without
+ * launching anything else when a list is bad; inside the kernels every index taken from a list or computed for a
+ * gather is range-checked before use, a bad one is skipped and recorded as FLOWMM_ERR_INDEX in the status word.
+ * Results of good inputs are the same as the release build's.
+ */
+int32_t flowmm_debug_build(void);
 
 /*
  * Profiling aid, per host thread, off by default.  While on, every compute entry point records

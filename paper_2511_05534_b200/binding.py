@@ -32,6 +32,7 @@ EXPORTS = (
     "flowmm_decode_workspace_bytes", "flowmm_decode_attention",
     "flowmm_full_flow_workspace_bytes", "flowmm_full_flow",
     "flowmm_merge_static_status", "flowmm_merge_static_poke_status",
+    "flowmm_recompress_workspace_bytes", "flowmm_recompress", "flowmm_debug_build",
 )
 
 
@@ -123,6 +124,9 @@ def load() -> ctypes.CDLL:
             getattr(lib, name).restype = ctypes.c_int
         lib.flowmm_merge_static.restype = ctypes.c_int
         lib.flowmm_merge_static_status.restype = ctypes.c_int
+        lib.flowmm_recompress_workspace_bytes.restype = ctypes.c_int
+        lib.flowmm_recompress.restype = ctypes.c_int
+        lib.flowmm_debug_build.restype = ctypes.c_int32
         lib.flowmm_merge_static_poke_status.restype = ctypes.c_int
         lib.flowmm_selftest_wait_timeout.restype = ctypes.c_int
         lib.flowmm_decode_workspace_bytes.restype = ctypes.c_int
@@ -247,6 +251,24 @@ def flowmm_compress_layer(p: Params, q_win, k, v, modality, k_out, v_out, ws, im
                                         ctypes.c_size_t(ws.numel()), _stream()), "flowmm_compress_layer")
 
 
+def flowmm_recompress_workspace_bytes(p: Params) -> int:
+    n = ctypes.c_size_t(0)
+    cp = p.c()
+    _check(load().flowmm_recompress_workspace_bytes(ctypes.byref(cp), ctypes.byref(n)), "flowmm_recompress_workspace_bytes")
+    return int(n.value)
+
+
+def flowmm_recompress(p: Params, q_win, k_cache, v_cache, row_modality, k_out, v_out, row_modality_out, ws,
+                      importance=None, rho=None, strategy=None, retained_idx=None, evicted_idx=None, match=None,
+                      match_sim=None):
+    """Section 3.3 again on a cache that grew during decoding; row_modality [units, kv_heads, rows] uint8."""
+    cp = p.c(q=q_win, k=k_cache, v=v_cache, ko=k_out, vo=v_out)
+    _check(load().flowmm_recompress(ctypes.byref(cp), _p(q_win), _p(k_cache), _p(v_cache), _p(row_modality), _p(k_out),
+                                    _p(v_out), _p(row_modality_out), _p(importance), _p(rho), _p(strategy),
+                                    _p(retained_idx), _p(evicted_idx), _p(match), _p(match_sim), _p(ws),
+                                    ctypes.c_size_t(ws.numel()), _stream()), "flowmm_recompress")
+
+
 def flowmm_last_device_status(ws) -> int:
     return int(load().flowmm_last_device_status(_p(ws), _stream()))
 
@@ -289,6 +311,10 @@ def flowmm_decode_attention(q, k, v, out, ws, softmax_scale: float = 0.0, path: 
 def flowmm_selftest_wait_timeout(ws):
     """Enqueue the kernel whose wait runs out; flowmm_last_device_status(ws) then reports TIMEOUT (8)."""
     _check(load().flowmm_selftest_wait_timeout(_p(ws), _stream()), "flowmm_selftest_wait_timeout")
+
+
+def flowmm_debug_build() -> bool:
+    return bool(load().flowmm_debug_build())
 
 
 def flowmm_last_launch_count() -> int:

@@ -8,6 +8,20 @@ namespace flowmm {
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegBig = -1.0e30f;   // "minus infinity" that stays finite under subtraction
+constexpr int kStatusIndex = 10;      // FLOWMM_ERR_INDEX
+
+// Range check of an index that is about to address memory.  In a build with -DFLOWMM_DEBUG a bad index is recorded
+// in the status word (first error wins) and reported to the caller, which skips the access; otherwise the check
+// compiles to nothing.
+#ifdef FLOWMM_DEBUG
+__device__ __forceinline__ bool index_ok(long long i, long long n, int *status) {
+    if (i >= 0 && i < n) return true;
+    if (status) atomicCAS(status, 0, kStatusIndex);
+    return false;
+}
+#else
+__device__ __forceinline__ constexpr bool index_ok(long long, long long, int *) { return true; }
+#endif
 
 // ---- element access -------------------------------------------------------------------------
 template <typename T> struct Elem;

@@ -56,6 +56,12 @@ inline void profile_mark(const char *name, cudaStream_t st) {
         profile_mark(name, st);                                        \
     } while (0)
 
+#define FLOWMM_TRY(expr)                         \
+    do {                                         \
+        const flowmm_status _s = (expr);         \
+        if (_s != FLOWMM_OK) return _s;          \
+    } while (0)
+
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // (unit, head) pairs per call: they index grid.x of several launches and 32-bit item counters
@@ -213,6 +219,48 @@ template <typename X> X *at(void *ws, size_t off) { return reinterpret_cast<X *>
 float tau_effective(const flowmm_params &p) {
     return p.tau_mode == FLOWMM_TAU_REL ? (float)((double)p.tau * (double)p.window / (double)p.seq_len) : p.tau;
 }
+
+// ---- debug build: the index lists a caller hands in are checked before any kernel uses them ---------
+#ifdef FLOWMM_DEBUG
+// One block per (unit, head): pivots and non-pivots inside [0, L) and strictly ascending, matches inside [-1, B).
+__global__ void debug_check_lists_kernel(const int32_t *retained, const int32_t *evicted, const int32_t *match,
+                                         int L, int B, int E, int *status) {
+    const int uh = blockIdx.x;
+    bool bad = false;
+    if (retained)
+        for (int s = threadIdx.x; s < B; s += blockDim.x) {
+            const int r = retained[(int64_t)uh * B + s];
+            bad |= r < 0 || r >= L || (s > 0 && retained[(int64_t)uh * B + s - 1] >= r);
+        }
+    if (evicted)
+        for (int j = threadIdx.x; j < E; j += blockDim.x) {
+            const int e = evicted[(int64_t)uh * E + j];
+            bad |= e < 0 || e >= L || (j > 0 && evicted[(int64_t)uh * E + j - 1] >= e);
+        }
+    if (match)
+        for (int j = threadIdx.x; j < E; j += blockDim.x) {
+            const int m = match[(int64_t)uh * E + j];
+            bad |= m < -1 || m >= B;
+        }
+    if (bad) atomicCAS(status, 0, kStatusIndex);
+}
+
+// Runs the check, waits for it and reports: the entry point launches nothing else when a list is bad.
+flowmm_status debug_check_lists(const flowmm_params &p, const int32_t *retained, const int32_t *evicted,
+                                const int32_t *match, int *status, cudaStream_t st) {
+    debug_check_lists_kernel<<<p.n_units * p.n_kv_heads, 256, 0, st>>>(retained, evicted, match, p.seq_len, p.n_keep,
+                                                                        p.seq_len - p.n_keep, status);
+    if (cudaGetLastError() != cudaSuccess) return FLOWMM_ERR_CUDA;
+    int32_t word = 0;
+    if (cudaMemcpyAsync(&word, status, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return FLOWMM_ERR_CUDA;
+    return word == kStatusIndex ? FLOWMM_ERR_INDEX : FLOWMM_OK;
+}
+#define FLOWMM_DEBUG_LISTS(p, ret, evi, mt, status, st) FLOWMM_TRY(debug_check_lists(p, ret, evi, mt, status, st))
+#else
+#define FLOWMM_DEBUG_LISTS(p, ret, evi, mt, status, st) do { } while (0)
+#endif
 
 // ---- step launchers (no validation; the entry points below validate) --------------------------
 
@@ -386,6 +434,7 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
     g.tau_eff = tau_effective(p);
     for (int i = 0; i < 3; ++i) g.ks[i] = p.k_stride[i];
     g.copy_here = y.c_tot <= 256;
+    g.status = at<int>(ws, y.status);
     // few heads: a head's lists are walked by more threads, the GPU is not full either way
     const int prep_threads = UH >= 4 * tc::sm_count() ? 256 : UH >= 2 * tc::sm_count() ? 512 : 1024;
     match_prepare_kernel<<<UH, prep_threads, 0, st>>>(g);
@@ -560,12 +609,6 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
     return FLOWMM_OK;
 }
 
-#define FLOWMM_TRY(expr)                         \
-    do {                                         \
-        const flowmm_status _s = (expr);         \
-        if (_s != FLOWMM_OK) return _s;          \
-    } while (0)
-
 }  // namespace
 
 extern "C" {
@@ -623,6 +666,7 @@ flowmm_status flowmm_match(const flowmm_params *p, const void *k, const float *i
     Layout y;
     FLOWMM_TRY(check_ws(p, ws, ws_bytes, y));
     FLOWMM_TRY(check_device());
+    FLOWMM_DEBUG_LISTS(*p, retained_idx, evicted_idx, nullptr, at<int>(ws, y.status), static_cast<cudaStream_t>(cuda_stream));
     return run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws,
                      static_cast<cudaStream_t>(cuda_stream));
 }
@@ -642,6 +686,7 @@ flowmm_status flowmm_merge(const flowmm_params *p, const void *k, const void *v,
     Layout y;
     FLOWMM_TRY(check_ws(p, ws, ws_bytes, y));
     FLOWMM_TRY(check_device());
+    FLOWMM_DEBUG_LISTS(*p, retained_idx, evicted_idx, match, at<int>(ws, y.status), static_cast<cudaStream_t>(cuda_stream));
     return run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws,
                      static_cast<cudaStream_t>(cuda_stream));
 }
@@ -693,10 +738,18 @@ flowmm_status flowmm_last_device_status(void *ws, void *cuda_stream) {
         if (cudaMemsetAsync(ws, 0, sizeof(word), st) != cudaSuccess) return FLOWMM_ERR_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return FLOWMM_ERR_CUDA;
     }
-    return word >= 0 && word <= FLOWMM_ERR_UNSUPPORTED_DEVICE ? static_cast<flowmm_status>(word) : FLOWMM_ERR_CUDA;
+    return word >= 0 && word <= FLOWMM_ERR_INDEX ? static_cast<flowmm_status>(word) : FLOWMM_ERR_CUDA;
 }
 
 int32_t flowmm_last_launch_count(void) { return g_launches; }
+
+int32_t flowmm_debug_build(void) {
+#ifdef FLOWMM_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 flowmm_status flowmm_profile_enable(int32_t on) {
     if (on && !g_prof.have_events) {
@@ -732,6 +785,7 @@ const char *flowmm_status_string(flowmm_status s) {
         case FLOWMM_ERR_CUDA: return "CUDA error";
         case FLOWMM_ERR_TIMEOUT: return "device-side wait timed out";
         case FLOWMM_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.x";
+        case FLOWMM_ERR_INDEX: return "index out of range (debug build)";
     }
     return "unknown status";
 }
@@ -1014,6 +1068,105 @@ extern "C" flowmm_status flowmm_decode_attention(const flowmm_decode_params *p, 
     return p->head_dim == 128 ? launch_decode<float, 128>(a, uh, n_q, st) : launch_decode<float, 64>(a, uh, n_q, st);
 }
 
+// ---- re-compression of a cache that grew during decoding ----------------------------------------
+namespace {
+
+// strategy of a unit copied to each of its KV heads (the per-head problems below take one strategy each)
+__global__ void expand_strategy_kernel(const int32_t *strategy, int n_units, int n_kv_heads, int32_t *per_head) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_units * n_kv_heads) per_head[i] = strategy[i / n_kv_heads];
+}
+
+// modality of the rows that were kept: out[uh, s] = row_modality[uh, retained[uh, s]]
+__global__ void gather_row_modality_kernel(const uint8_t *row_modality, const int32_t *retained, int64_t n, int L, int B,
+                                           uint8_t *out) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = row_modality[(i / B) * L + retained[i]];
+}
+
+// Every (unit, KV head) of the cache as a problem of its own: one KV head, its G query heads, its own row modalities.
+// Needs the unit stride of every tensor to be heads x head stride (one stride then steps through units and heads).
+bool per_head_params(const flowmm_params &p, flowmm_params &ph) {
+    const int G = p.n_q_heads / p.n_kv_heads;
+    if (p.q_stride[0] != (int64_t)p.n_q_heads * p.q_stride[1] || p.k_stride[0] != (int64_t)p.n_kv_heads * p.k_stride[1] ||
+        p.v_stride[0] != (int64_t)p.n_kv_heads * p.v_stride[1] || p.ko_stride[0] != (int64_t)p.n_kv_heads * p.ko_stride[1] ||
+        p.vo_stride[0] != (int64_t)p.n_kv_heads * p.vo_stride[1])
+        return false;
+    ph = p;
+    ph.n_units = p.n_units * p.n_kv_heads; ph.n_q_heads = G; ph.n_kv_heads = 1;
+    ph.q_stride[0] = (int64_t)G * p.q_stride[1];
+    ph.k_stride[0] = p.k_stride[1]; ph.v_stride[0] = p.v_stride[1];
+    ph.ko_stride[0] = p.ko_stride[1]; ph.vo_stride[0] = p.vo_stride[1];
+    return true;
+}
+
+struct RecompressLayout { size_t strategy_h, total; };
+RecompressLayout recompress_layout(const flowmm_params &ph) {
+    RecompressLayout r;
+    r.strategy_h = align256(make_layout(ph).total);
+    r.total = r.strategy_h + align256((size_t)ph.n_units * 4);
+    return r;
+}
+
+}  // namespace
+
+extern "C" flowmm_status flowmm_recompress_workspace_bytes(const flowmm_params *p, size_t *bytes) {
+    if (!bytes) return FLOWMM_ERR_NULL;
+    FLOWMM_TRY(validate(p));
+    flowmm_params ph;
+    if (!per_head_params(*p, ph)) return FLOWMM_ERR_ALIGN;
+    FLOWMM_TRY(validate(&ph));
+    *bytes = recompress_layout(ph).total;
+    return FLOWMM_OK;
+}
+
+extern "C" flowmm_status flowmm_recompress(const flowmm_params *p, const void *q_win, const void *k_cache,
+                                           const void *v_cache, const uint8_t *row_modality, void *k_out, void *v_out,
+                                           uint8_t *row_modality_out, float *importance, float *rho, int32_t *strategy,
+                                           int32_t *retained_idx, int32_t *evicted_idx, int32_t *match, float *match_sim,
+                                           void *ws, size_t ws_bytes, void *cuda_stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    profile_begin(st);
+    FLOWMM_TRY(validate(p));
+    if (!q_win || !k_cache || !v_cache || !row_modality || !k_out || !v_out || !row_modality_out) return FLOWMM_ERR_NULL;
+    if (!aligned16(q_win) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_out) || !aligned16(v_out) ||
+        !strides_ok(p->q_stride, p->head_dim) || !strides_ok(p->k_stride, p->head_dim) ||
+        !strides_ok(p->v_stride, p->head_dim) || !strides_ok(p->ko_stride, p->head_dim) ||
+        !strides_ok(p->vo_stride, p->head_dim))
+        return FLOWMM_ERR_ALIGN;
+    flowmm_params ph;
+    if (!per_head_params(*p, ph)) return FLOWMM_ERR_ALIGN;
+    FLOWMM_TRY(validate(&ph));
+    if (!ws) return FLOWMM_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(ws) & 255) return FLOWMM_ERR_ALIGN;
+    const Layout y = make_layout(ph);
+    const RecompressLayout r = recompress_layout(ph);
+    if (ws_bytes < r.total) return FLOWMM_ERR_WORKSPACE;
+    FLOWMM_TRY(check_device());
+    if (!importance) importance = at<float>(ws, y.importance);
+    if (!rho) rho = at<float>(ws, y.rho);
+    if (!strategy) strategy = at<int32_t>(ws, y.strategy);
+    if (!retained_idx) retained_idx = at<int32_t>(ws, y.retained);
+    if (!evicted_idx) evicted_idx = at<int32_t>(ws, y.evicted);
+    if (!match) match = at<int32_t>(ws, y.match);
+    if (!match_sim) match_sim = at<float>(ws, y.match_sim);
+    float *cross_mass = at<float>(ws, y.cross_mass);             // [U * Hkv, G] = [U, Hq]
+    int32_t *strategy_h = at<int32_t>(ws, r.strategy_h);
+    // scoring per (unit, KV head) against that head's own row modalities; Eq. 6 over all query heads of the layer
+    FLOWMM_TRY(run_score(ph, y, q_win, k_cache, row_modality, importance, cross_mass, ws, st));
+    FLOWMM_TRY(run_layer_flow(*p, cross_mass, rho, strategy, st));
+    expand_strategy_kernel<<<(ph.n_units + 255) / 256, 256, 0, st>>>(strategy, p->n_units, p->n_kv_heads, strategy_h);
+    FLOWMM_LAUNCHED("expand_strategy");
+    FLOWMM_TRY(run_select(ph, importance, retained_idx, evicted_idx, st));
+    FLOWMM_TRY(run_match(ph, y, k_cache, importance, row_modality, retained_idx, evicted_idx, strategy_h, match, match_sim, ws, st));
+    FLOWMM_TRY(run_merge(ph, y, k_cache, v_cache, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws, st));
+    const int64_t n = (int64_t)ph.n_units * p->n_keep;
+    gather_row_modality_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(row_modality, retained_idx, n, p->seq_len, p->n_keep,
+                                                                            row_modality_out);
+    FLOWMM_LAUNCHED("gather_row_modality");
+    return FLOWMM_OK;
+}
+
 // ---- bounded-wait self-test ----------------------------------------------------------------------
 namespace {
 // One CTA waits on an mbarrier phase that nothing completes, with the same bounded wait the
@@ -1099,6 +1252,7 @@ extern "C" flowmm_status flowmm_merge_static(const flowmm_params *p, const void 
     FLOWMM_TRY(check_device());
     void *base = nullptr;
     FLOWMM_TRY(merge_static_base(&base));
+    FLOWMM_DEBUG_LISTS(*p, retained_idx, evicted_idx, match, static_cast<int *>(base), static_cast<cudaStream_t>(cuda_stream));
     // Nothing in this scratch has to start at zero: the slot lists, the piece table, the work counter and
     // the arrival counters are written (or cleared) by this call's first kernel before they are read, a
     // partial-sum record is only read for pieces that wrote it in the same call, and the status word is

@@ -219,7 +219,7 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                         if (w.y == best) idx = 4 * q4 + 1;
                         if (w.x == best) idx = 4 * q4;
                     }
-                    return __float_as_int(tc::lds32(md + slot_off + (best_cc + idx) * 4));
+                    return index_ok(best_cc + idx, N, A.status) ? __float_as_int(tc::lds32(md + slot_off + (best_cc + idx) * 4)) : -1;
                 };
                 const int park_blk = intra ? -1 : (t0 >> 4);
                 for (int blk = 0; blk < nb_all; ++blk) {
@@ -261,7 +261,7 @@ match_small_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 if (lane == 0) tc::mbar_arrive(bar(kBarSetFree + team));   // this warp has read the accumulator
                 int slot = resolve();
                 if (match_better(val_a, slot_a, best, slot)) { best = val_a; slot = slot_a; }
-                if (in_range && my_rank >= 0 && ok) {                // a non-pivot: report its match
+                if (in_range && my_rank >= 0 && ok && index_ok(my_rank, A.E, A.status)) {   // a non-pivot: report its match
                     float sim = 0.f;
                     if (slot >= 0 && ssq > 0.f) sim = best * rsqrtf(ssq);
                     A.match[(int64_t)uh * A.E + my_rank] = slot;

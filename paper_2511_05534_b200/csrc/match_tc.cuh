@@ -32,6 +32,7 @@ struct MatchPrepArgs {
     int *rank;                   // [UH, L]  position in the non-pivot list, or -(s + 2) for the pivot of slot s
     uint8_t *tile_mod;           // [U, n_rt] per tile of 256 tokens; bit 0: holds text tokens, bit 1: visual tokens
     int Hkv, L, B, E, Ctot, n_rt;
+    int *status;                 // device status word (index checks of the debug build report here)
     int copy_here;               // 1: this kernel also gathers the candidate rows; 0: match_gather_kernel does
     float tau_eff;
     int64_t ks[3];
@@ -51,7 +52,8 @@ __device__ __forceinline__ void match_gather_rows(const MatchPrepArgs &A, int uh
     for (int pos = lo + (tid >> 4); pos < hi; pos += nthreads >> 4) {       // uniform trip count within a warp
         const int s = slot_out[pos];
         uint4 val = make_uint4(0, 0, 0, 0);
-        if (s >= 0) val = *reinterpret_cast<const uint4 *>(kb + (int64_t)ret[s] * A.ks[2] + sub * 8);
+        if (s >= 0 && index_ok(s, A.B, A.status) && index_ok(ret[s], A.L, A.status))
+            val = *reinterpret_cast<const uint4 *>(kb + (int64_t)ret[s] * A.ks[2] + sub * 8);
         dst[(int64_t)pos * 16 + sub] = val;
         float x[8], ssq = 0.f;
         Elem<__nv_bfloat16>::unpack(val, x);
@@ -77,8 +79,10 @@ __global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs
     float *scale_out = A.cand_scale + (int64_t)uh * A.Ctot;
 
     for (int i = tid; i < A.Ctot; i += blockDim.x) { slot_out[i] = -1; scale_out[i] = __int_as_float(0x7FC00000); }   // NaN: no candidate here
-    for (int s = tid; s < A.B; s += blockDim.x) rank[ret[s]] = -(s + 2);
-    for (int j = tid; j < A.E; j += blockDim.x) rank[evi[j]] = j;
+    for (int s = tid; s < A.B; s += blockDim.x)
+        if (index_ok(ret[s], A.L, A.status)) rank[ret[s]] = -(s + 2);
+    for (int j = tid; j < A.E; j += blockDim.x)
+        if (index_ok(evi[j], A.L, A.status)) rank[evi[j]] = j;
     if (h == 0) {
         for (int t = tid; t < A.n_rt; t += blockDim.x) {
             int bits = 0;
@@ -90,7 +94,7 @@ __global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs
     // admissible text pivots first: count them to know where the visual group starts
     int n_text = 0;
     for (int s = tid; s < A.B; s += blockDim.x) {
-        const int r = ret[s];
+        const int r = index_ok(ret[s], A.L, A.status) ? ret[s] : 0;
         n_text += (imp[r] <= A.tau_eff && mod[r] == 0) ? 1 : 0;
     }
     int total;
@@ -103,7 +107,7 @@ __global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs
         const int s = base + tid;
         int ft = 0, fv = 0, r = 0;
         if (s < A.B) {
-            r = ret[s];
+            r = index_ok(ret[s], A.L, A.status) ? ret[s] : 0;
             const bool adm = imp[r] <= A.tau_eff;              // Eq. 10: pivots above tau are kept out of merging
             ft = adm && mod[r] == 0;
             fv = adm && mod[r] != 0;
@@ -371,7 +375,8 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             float ssq = 0.f;                                         // squared norm of this row's key, this warp's half of it
             auto resolve = [&]() -> int {                            // slot of the running winner
                 if (win < 0) return -1;
-                return slots[p.lo + best_tile * kMtCols + (b0 + (win >> 4)) * 16 + 15 - (win & 15)];
+                const int col = p.lo + best_tile * kMtCols + (b0 + (win >> 4)) * 16 + 15 - (win & 15);
+                return index_ok(col, A.Ctot, A.status) ? slots[col] : -1;
             };
             auto park = [&](int t) {
                 if (best > before) best_tile = t;                   // the winner may be of this tile's earlier blocks
@@ -473,7 +478,7 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 ssq += other.z;
                 if (in_range) {
                     const int j = my_rank;
-                    if (j >= 0) {                                    // a non-pivot: report its match
+                    if (j >= 0 && index_ok(j, A.E, A.status)) {      // a non-pivot: report its match
                         float sim = 0.f;
                         if (slot >= 0 && ssq > 0.f) sim = best * rsqrtf(ssq);
                         A.match[(int64_t)p.uh * A.E + j] = slot;

@@ -104,6 +104,7 @@ __global__ void __launch_bounds__(kThreads, 3) merge_staged_kernel(const MergeAr
         int tok = t < 32 ? tok_a : tok_b;
         bool go = rowslot >= 1 && rowslot <= n_mem;
         if (rowslot == 0) { tok = pc.r; go = pivot; }
+        if (go && !index_ok(tok, A.L, status)) tok = 0;     // (debug build: a bad row number is recorded; row 0 stands in so that the byte count still arrives)
         if (go) tc::bulk_load(buf + rowslot * kRowBytes + (is_v ? 256u : 0u), src_base + (int64_t)tok * tstride, 256u, bar);
     };
 
