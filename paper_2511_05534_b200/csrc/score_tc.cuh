@@ -238,6 +238,63 @@ __global__ void score_combine_kernel(const float2 *row_part, int n_chunk, int GW
     negc[i] = out;
 }
 
+// The common case of pass 2's inner step, written out in PTX so that it costs what it must and no more: 32 accumulator
+// columns of this thread's key (32 proxy rows of one query head): probability = 2^(logit * scale + row constant), with
+// the row constants read as packed pairs from shared memory, the multiply-adds and the additions as packed pairs, one
+// exp2 per element; returns the sum of the 32 probabilities.  No mask and no split by modality: chunks that need either
+// take the general path.
+//   taddr  TMEM address of the chunk for this warp's lanes     negc  shared address of its 32 row constants
+// (three phases, so that no exponential's result is needed before the last one has been issued: logits in place,
+// exponentials in place, then a tree of packed additions)
+#define FLOWMM_CS_X(q, i0, i1, i2, i3)                                                      \
+    "ld.shared.v2.b64 {n0, n1}, [%2 + " #q " * 16];\n\t"                                    \
+    "mov.b64 x0, {a" #i0 ", a" #i1 "};\n\t"                                                 \
+    "mov.b64 x1, {a" #i2 ", a" #i3 "};\n\t"                                                 \
+    "fma.rn.f32x2 x0, x0, sc, n0;\n\t"                                                      \
+    "fma.rn.f32x2 x1, x1, sc, n1;\n\t"                                                      \
+    "mov.b64 {a" #i0 ", a" #i1 "}, x0;\n\t"                                                 \
+    "mov.b64 {a" #i2 ", a" #i3 "}, x1;\n\t"
+#define FLOWMM_CS_E(i) "ex2.approx.ftz.f32 a" #i ", a" #i ";\n\t"
+#define FLOWMM_CS_P(k, i0, i1) "mov.b64 p" #k ", {a" #i0 ", a" #i1 "};\n\t"
+#define FLOWMM_CS_A(d, x, y) "add.rn.f32x2 p" #d ", p" #x ", p" #y ";\n\t"
+__device__ __forceinline__ float colsum_chunk32(uint32_t taddr, uint32_t negc, float scale_log2) {
+    float csum;
+    asm volatile(
+        "{\n\t"
+        ".reg .b32 a<32>;\n\t"
+        ".reg .b64 n0, n1, x0, x1, sc, p<16>;\n\t"
+        ".reg .f32 f0, f1;\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {a0, a1, a2, a3, a4, a5, a6, a7, a8, a9, a10, a11, a12, a13, a14, a15, "
+        "a16, a17, a18, a19, a20, a21, a22, a23, a24, a25, a26, a27, a28, a29, a30, a31}, [%1];\n\t"
+        "mov.b64 sc, {%3, %3};\n\t"
+        "tcgen05.wait::ld.sync.aligned;\n\t"
+        FLOWMM_CS_X(0, 0, 1, 2, 3) FLOWMM_CS_X(1, 4, 5, 6, 7) FLOWMM_CS_X(2, 8, 9, 10, 11) FLOWMM_CS_X(3, 12, 13, 14, 15)
+        FLOWMM_CS_X(4, 16, 17, 18, 19) FLOWMM_CS_X(5, 20, 21, 22, 23) FLOWMM_CS_X(6, 24, 25, 26, 27) FLOWMM_CS_X(7, 28, 29, 30, 31)
+        FLOWMM_CS_E(0) FLOWMM_CS_E(1) FLOWMM_CS_E(2) FLOWMM_CS_E(3) FLOWMM_CS_E(4) FLOWMM_CS_E(5) FLOWMM_CS_E(6) FLOWMM_CS_E(7)
+        FLOWMM_CS_E(8) FLOWMM_CS_E(9) FLOWMM_CS_E(10) FLOWMM_CS_E(11) FLOWMM_CS_E(12) FLOWMM_CS_E(13) FLOWMM_CS_E(14) FLOWMM_CS_E(15)
+        FLOWMM_CS_E(16) FLOWMM_CS_E(17) FLOWMM_CS_E(18) FLOWMM_CS_E(19) FLOWMM_CS_E(20) FLOWMM_CS_E(21) FLOWMM_CS_E(22) FLOWMM_CS_E(23)
+        FLOWMM_CS_E(24) FLOWMM_CS_E(25) FLOWMM_CS_E(26) FLOWMM_CS_E(27) FLOWMM_CS_E(28) FLOWMM_CS_E(29) FLOWMM_CS_E(30) FLOWMM_CS_E(31)
+        FLOWMM_CS_P(0, 0, 1) FLOWMM_CS_P(1, 2, 3) FLOWMM_CS_P(2, 4, 5) FLOWMM_CS_P(3, 6, 7) FLOWMM_CS_P(4, 8, 9) FLOWMM_CS_P(5, 10, 11)
+        FLOWMM_CS_P(6, 12, 13) FLOWMM_CS_P(7, 14, 15) FLOWMM_CS_P(8, 16, 17) FLOWMM_CS_P(9, 18, 19) FLOWMM_CS_P(10, 20, 21)
+        FLOWMM_CS_P(11, 22, 23) FLOWMM_CS_P(12, 24, 25) FLOWMM_CS_P(13, 26, 27) FLOWMM_CS_P(14, 28, 29) FLOWMM_CS_P(15, 30, 31)
+        FLOWMM_CS_A(0, 0, 1) FLOWMM_CS_A(2, 2, 3) FLOWMM_CS_A(4, 4, 5) FLOWMM_CS_A(6, 6, 7) FLOWMM_CS_A(8, 8, 9) FLOWMM_CS_A(10, 10, 11)
+        FLOWMM_CS_A(12, 12, 13) FLOWMM_CS_A(14, 14, 15)
+        FLOWMM_CS_A(0, 0, 2) FLOWMM_CS_A(4, 4, 6) FLOWMM_CS_A(8, 8, 10) FLOWMM_CS_A(12, 12, 14)
+        FLOWMM_CS_A(0, 0, 4) FLOWMM_CS_A(8, 8, 12)
+        FLOWMM_CS_A(0, 0, 8)
+        "mov.b64 {f0, f1}, p0;\n\t"
+        "add.f32 %0, f0, f1;\n\t"
+        "}"
+        : "=f"(csum)
+        : "r"(taddr), "r"(negc), "f"(scale_log2)
+        : "memory");
+    return csum;
+}
+#undef FLOWMM_CS_X
+#undef FLOWMM_CS_E
+#undef FLOWMM_CS_P
+#undef FLOWMM_CS_A
+
 // ---------------------------------------------------------------------------------------------
 // Pass 2.  item = (unit*head, tile of 256 keys); the B stream is the head group's proxy rows.
 template <class S>
@@ -270,6 +327,7 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
         const uint32_t xch = c.epi_addr() + row * 4;            // hand-over slot of this row
         const uint32_t pxch = c.partner_addr() + row * 4;
         int k = 0, bt = 0, cached_u = -1;
+        const int w_shift = 31 - __clz(A.W);
         uint32_t wbits[4] = {0, 0, 0, 0};                            // modality of the proxy tokens, 32 per word
         bool ok = true;
         for (int item = blockIdx.x; ok && item < A.n_items2; item += gridDim.x) {
@@ -303,9 +361,11 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                 ok = S::extra_wait(c, bt, A.status) && S::acc_wait(c, k, A.status);
                 if (!ok) break;
                 const uint32_t negc4 = c.extra(bt);
-                S::for_each_chunk(c, (ncols + 31) >> 5, [&](int ch, uint32_t (&acc)[32]) {
+                constexpr int kPerC = S::kCols / 64;               // 32-column chunks a warp takes of a full tile
+                const int chunk_hi = min((ncols + 31) >> 5, kPerC * c.colhalf + kPerC);
+                for (int ch = kPerC * c.colhalf; ch < chunk_hi; ++ch) {
                     const int col = t * S::kCols + ch * 32;        // proxy row index r = g_local * W + a
-                    const int g_local = col / A.W, a0 = col % A.W;
+                    const int g_local = col >> w_shift, a0 = col & (A.W - 1);   // (the window is 32, 64 or 128 rows)
                     if (g_local != cur_g) {                          // a head is complete: publish its mass
                         if (cur_g >= 0) {
                             const float tot = warp_sum(cg);
@@ -314,6 +374,21 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                         cg = 0.f;
                         cur_g = g_local;
                     }
+                    // proxy tokens of the other modality than this key's
+                    const uint32_t wm = a0 < 32 ? wbits[0] : a0 < 64 ? wbits[1] : a0 < 96 ? wbits[2] : wbits[3];
+                    const uint32_t other = my_vis ? ~wm : wm;
+                    // the common case: no causal mask inside this tile, and the chunk's proxy tokens are all of this
+                    // key's modality or all of the other one (decided for the whole warp: the TMEM read is warp-wide)
+                    const bool plain = !masked_tile && (other == 0u || other == 0xFFFFFFFFu);
+                    if (__all_sync(0xFFFFFFFFu, plain)) {
+                        const float csum = colsum_chunk32(S::acc_addr(c, ch), negc4 + ch * 128, A.scale_log2);
+                        imp += csum;
+                        cg += other != 0u ? csum : 0.f;
+                        continue;
+                    }
+                    uint32_t acc[32];
+                    tc::tmem_ld32(S::acc_addr(c, ch), acc);
+                    tc::tmem_ld_wait(acc);
                     float pr[32];
                     const float2 sc2 = make_float2(A.scale_log2, A.scale_log2);
 #pragma unroll
@@ -340,9 +415,6 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                     }
                     const float csum = (s01.x + s01.y) + (s23.x + s23.y);
                     imp += csum;
-                    // proxy tokens of the other modality than this key's
-                    const uint32_t wm = a0 < 32 ? wbits[0] : a0 < 64 ? wbits[1] : a0 < 96 ? wbits[2] : wbits[3];
-                    const uint32_t other = my_vis ? ~wm : wm;
                     if (other == 0xFFFFFFFFu) cg += csum;
                     else if (other != 0u) {
                         float x = 0.f;
@@ -350,7 +422,7 @@ score_colsum_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_c
                         for (int j = 0; j < 32; ++j) x += ((other >> j) & 1u) ? pr[j] : 0.f;
                         cg += x;
                     }
-                });
+                }
                 S::acc_release(c);
             }
             if (ok && cur_g >= 0) {
