@@ -206,7 +206,7 @@ KERNEL_MODEL = {   # kernel name -> entry of kernel_model()
 
 # Share of a scoring kernel's exponentials that it evaluates as a polynomial on the FMA pipe (the kernels' own
 # constants: score_tc.cuh); the rest goes through the exp2 unit.
-EXP_FMA_SHARE = {"score_stats_tc": 0.25, "score_colsum_tc": 0.0}
+EXP_FMA_SHARE = {"score_stats_tc": 0.25, "score_colsum_tc": 0.25}
 
 
 def model_for(name, model):

@@ -129,11 +129,16 @@ score_stats_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
                                 const float2 neg2 = make_float2(-mx, -mx), sc2 = make_float2(A.scale_log2, A.scale_log2);
                                 float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
 #pragma unroll
-                                for (int j = 0; j < 32; j += 4) {
+                                for (int j = 0; j < 32; j += 8) {        // every fourth exponential on the FMA pipe, two at a time
                                     const float2 x01 = tc::ffma2(make_float2(raw[j], raw[j + 1]), sc2, neg2);
                                     const float2 x23 = tc::ffma2(make_float2(raw[j + 2], raw[j + 3]), sc2, neg2);
+                                    const float2 x45 = tc::ffma2(make_float2(raw[j + 4], raw[j + 5]), sc2, neg2);
+                                    const float2 x67 = tc::ffma2(make_float2(raw[j + 6], raw[j + 7]), sc2, neg2);
+                                    const float2 pf = tc::ex2_fma2(make_float2(x23.y, x67.y));
                                     a01 = tc::fadd2(a01, make_float2(tc::ex2(x01.x), tc::ex2(x01.y)));
-                                    a23 = tc::fadd2(a23, make_float2(tc::ex2(x23.x), tc::ex2_fma(x23.y)));   // every fourth one on the FMA pipe
+                                    a23 = tc::fadd2(a23, make_float2(tc::ex2(x23.x), pf.x));
+                                    a01 = tc::fadd2(a01, make_float2(tc::ex2(x45.x), tc::ex2(x45.y)));
+                                    a23 = tc::fadd2(a23, make_float2(tc::ex2(x67.x), pf.y));
                                 }
                                 add0 = a01.x; add1 = a01.y; add2 = a23.x; add3 = a23.y;
                                 if constexpr (kFlow) {
@@ -255,6 +260,24 @@ __global__ void score_combine_kernel(const float2 *row_part, int n_chunk, int GW
     "mov.b64 {a" #i0 ", a" #i1 "}, x0;\n\t"                                                 \
     "mov.b64 {a" #i2 ", a" #i3 "}, x1;\n\t"
 #define FLOWMM_CS_E(i) "ex2.approx.ftz.f32 a" #i ", a" #i ";\n\t"
+// 2^x for the pair (a_i, a_j) on the FMA pipe instead of the exp2 unit (which sets this step's pace): x clamped at
+// -125, n = round(x) by the 1.5 * 2^23 trick, 2^f on f = x - n in [-0.5, 0.5] by a degree-4 polynomial (own least-squares
+// fit at Chebyshev nodes with the constant fixed at 1: relative error 3.6e-6), n added to the exponent field.
+#define FLOWMM_CS_POLY(i, j)                                                          \
+    "max.f32 a" #i ", a" #i ", 0fC2FA0000;\n\t"                                        \
+    "max.f32 a" #j ", a" #j ", 0fC2FA0000;\n\t"                                        \
+    "mov.b64 x0, {a" #i ", a" #j "};\n\t"                                              \
+    "add.rn.f32x2 x1, x0, kmg;\n\t"          /* t = x + 1.5 * 2^23 */                  \
+    "mov.b64 {f0, f1}, x1;\n\t"                                                       \
+    "sub.rn.f32x2 x1, x1, kmg;\n\t"          /* n */                                   \
+    "sub.rn.f32x2 x0, x0, x1;\n\t"           /* f */                                   \
+    "fma.rn.f32x2 x1, kc4, x0, kc3;\n\t"                                              \
+    "fma.rn.f32x2 x1, x1, x0, kc2;\n\t"                                               \
+    "fma.rn.f32x2 x1, x1, x0, kc1;\n\t"                                               \
+    "fma.rn.f32x2 x1, x1, x0, kone;\n\t"                                              \
+    "mov.b64 {a" #i ", a" #j "}, x1;\n\t"                                              \
+    "mad.lo.s32 a" #i ", f0, 8388608, a" #i ";\n\t"                                    \
+    "mad.lo.s32 a" #j ", f1, 8388608, a" #j ";\n\t"
 #define FLOWMM_CS_P(k, i0, i1) "mov.b64 p" #k ", {a" #i0 ", a" #i1 "};\n\t"
 #define FLOWMM_CS_A(d, x, y) "add.rn.f32x2 p" #d ", p" #x ", p" #y ";\n\t"
 __device__ __forceinline__ float colsum_chunk32(uint32_t taddr, uint32_t negc, float scale_log2) {
@@ -262,18 +285,25 @@ __device__ __forceinline__ float colsum_chunk32(uint32_t taddr, uint32_t negc, f
     asm volatile(
         "{\n\t"
         ".reg .b32 a<32>;\n\t"
-        ".reg .b64 n0, n1, x0, x1, sc, p<16>;\n\t"
-        ".reg .f32 f0, f1;\n\t"
+        ".reg .b64 n0, n1, x0, x1, sc, p<16>, kmg, kc1, kc2, kc3, kc4, kone;\n\t"
+        ".reg .b32 f0, f1;\n\t"
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 {a0, a1, a2, a3, a4, a5, a6, a7, a8, a9, a10, a11, a12, a13, a14, a15, "
         "a16, a17, a18, a19, a20, a21, a22, a23, a24, a25, a26, a27, a28, a29, a30, a31}, [%1];\n\t"
         "mov.b64 sc, {%3, %3};\n\t"
+        "mov.b64 kmg, 0x4B4000004B400000;\n\t"      /* 12582912.0f twice */
+        "mov.b64 kone, 0x3F8000003F800000;\n\t"
+        "mov.b64 kc1, 0x3F3170613F317061;\n\t"      /* 0.69312102 */
+        "mov.b64 kc2, 0x3E75FCD43E75FCD4;\n\t"      /* 0.24022228 */
+        "mov.b64 kc3, 0x3D650E813D650E81;\n\t"      /* 0.05592204 */
+        "mov.b64 kc4, 0x3C1E78073C1E7807;\n\t"      /* 0.00967217 */
         "tcgen05.wait::ld.sync.aligned;\n\t"
         FLOWMM_CS_X(0, 0, 1, 2, 3) FLOWMM_CS_X(1, 4, 5, 6, 7) FLOWMM_CS_X(2, 8, 9, 10, 11) FLOWMM_CS_X(3, 12, 13, 14, 15)
         FLOWMM_CS_X(4, 16, 17, 18, 19) FLOWMM_CS_X(5, 20, 21, 22, 23) FLOWMM_CS_X(6, 24, 25, 26, 27) FLOWMM_CS_X(7, 28, 29, 30, 31)
-        FLOWMM_CS_E(0) FLOWMM_CS_E(1) FLOWMM_CS_E(2) FLOWMM_CS_E(3) FLOWMM_CS_E(4) FLOWMM_CS_E(5) FLOWMM_CS_E(6) FLOWMM_CS_E(7)
-        FLOWMM_CS_E(8) FLOWMM_CS_E(9) FLOWMM_CS_E(10) FLOWMM_CS_E(11) FLOWMM_CS_E(12) FLOWMM_CS_E(13) FLOWMM_CS_E(14) FLOWMM_CS_E(15)
-        FLOWMM_CS_E(16) FLOWMM_CS_E(17) FLOWMM_CS_E(18) FLOWMM_CS_E(19) FLOWMM_CS_E(20) FLOWMM_CS_E(21) FLOWMM_CS_E(22) FLOWMM_CS_E(23)
-        FLOWMM_CS_E(24) FLOWMM_CS_E(25) FLOWMM_CS_E(26) FLOWMM_CS_E(27) FLOWMM_CS_E(28) FLOWMM_CS_E(29) FLOWMM_CS_E(30) FLOWMM_CS_E(31)
+        // every fourth exponential goes to the FMA pipe, placed between the others
+        FLOWMM_CS_E(0) FLOWMM_CS_E(1) FLOWMM_CS_E(2) FLOWMM_CS_E(4) FLOWMM_CS_E(5) FLOWMM_CS_E(6) FLOWMM_CS_POLY(3, 7)
+        FLOWMM_CS_E(8) FLOWMM_CS_E(9) FLOWMM_CS_E(10) FLOWMM_CS_E(12) FLOWMM_CS_E(13) FLOWMM_CS_E(14) FLOWMM_CS_POLY(11, 15)
+        FLOWMM_CS_E(16) FLOWMM_CS_E(17) FLOWMM_CS_E(18) FLOWMM_CS_E(20) FLOWMM_CS_E(21) FLOWMM_CS_E(22) FLOWMM_CS_POLY(19, 23)
+        FLOWMM_CS_E(24) FLOWMM_CS_E(25) FLOWMM_CS_E(26) FLOWMM_CS_E(28) FLOWMM_CS_E(29) FLOWMM_CS_E(30) FLOWMM_CS_POLY(27, 31)
         FLOWMM_CS_P(0, 0, 1) FLOWMM_CS_P(1, 2, 3) FLOWMM_CS_P(2, 4, 5) FLOWMM_CS_P(3, 6, 7) FLOWMM_CS_P(4, 8, 9) FLOWMM_CS_P(5, 10, 11)
         FLOWMM_CS_P(6, 12, 13) FLOWMM_CS_P(7, 14, 15) FLOWMM_CS_P(8, 16, 17) FLOWMM_CS_P(9, 18, 19) FLOWMM_CS_P(10, 20, 21)
         FLOWMM_CS_P(11, 22, 23) FLOWMM_CS_P(12, 24, 25) FLOWMM_CS_P(13, 26, 27) FLOWMM_CS_P(14, 28, 29) FLOWMM_CS_P(15, 30, 31)
@@ -292,6 +322,7 @@ __device__ __forceinline__ float colsum_chunk32(uint32_t taddr, uint32_t negc, f
 }
 #undef FLOWMM_CS_X
 #undef FLOWMM_CS_E
+#undef FLOWMM_CS_POLY
 #undef FLOWMM_CS_P
 #undef FLOWMM_CS_A
 
