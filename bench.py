@@ -49,6 +49,7 @@ def parse_args():
                     help="--impl reference: wall time its warm-up and timed steps may spend together")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="skip the decode-attention timing over the caches")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (host buffers), e.g. under a profiler")
     ap.add_argument("--cpu-baseline-units", type=int, default=0)
     return ap.parse_args()
 
@@ -526,7 +527,7 @@ def run_ours(args):
 
 
     try:
-        e2e = end_to_end()
+        e2e = {"value": None, "unit": UNIT, "skipped": "--no-e2e"} if args.no_e2e else end_to_end()
     except (RuntimeError, MemoryError) as exc:      # e.g. the host cannot pin a whole input set: say so, keep the line
         if "device status" in str(exc):
             raise
