@@ -210,21 +210,22 @@ __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) 
 //   taddr   TMEM address of the block for this warp's lanes        scales   shared address of the block's 16 norms
 // (TMEM is read 32 columns at a time: a read has a cost of its own that does not shrink with its width, and sixteen
 // warps reading 16 columns each time kept the tensor core waiting for its accumulators.)
-#define FLOWMM_MB_MUL2(i, j, k, ti, tj)                                                                        \
+#define FLOWMM_MB_MUL2(i, j, k, ti, tj, MASK)                                                                  \
     "mov.b64 t0, {a" #i ", a" #j "};\n\tmul.rn.f32x2 t0, t0, s" #k ";\n\tmov.b64 {a" #i ", a" #j "}, t0;\n\t"    \
-    "lop3.b32 a" #i ", a" #i ", 0xFFFFFFF0, " #ti ", 0xEA;\n\t"                                                \
-    "lop3.b32 a" #j ", a" #j ", 0xFFFFFFF0, " #tj ", 0xEA;\n\t"
+    "lop3.b32 a" #i ", a" #i ", " MASK ", " #ti ", 0xEA;\n\t"                                                   \
+    "lop3.b32 a" #j ", a" #j ", " MASK ", " #tj ", 0xEA;\n\t"
 #define FLOWMM_MB_LDS(OFF)                                     \
     "ld.shared.v2.b64 {s0, s1}, [%3 + " #OFF "];\n\t"          \
     "ld.shared.v2.b64 {s2, s3}, [%3 + " #OFF " + 16];\n\t"     \
     "ld.shared.v2.b64 {s4, s5}, [%3 + " #OFF " + 32];\n\t"     \
     "ld.shared.v2.b64 {s6, s7}, [%3 + " #OFF " + 48];\n\t"
 // 16 columns held in registers a<c0> .. a<c15>: products, tags, maximum, comparison with the running maximum;
-// WIN = 16 x block number, as an asm operand reference
-#define FLOWMM_MB_STEP(c0, c1, c2, c3, c4, c5, c6, c7, c8, c9, c10, c11, c12, c13, c14, c15, WIN)               \
-    FLOWMM_MB_MUL2(c0, c1, 0, 15, 14) FLOWMM_MB_MUL2(c2, c3, 1, 13, 12) FLOWMM_MB_MUL2(c4, c5, 2, 11, 10)       \
-    FLOWMM_MB_MUL2(c6, c7, 3, 9, 8) FLOWMM_MB_MUL2(c8, c9, 4, 7, 6) FLOWMM_MB_MUL2(c10, c11, 5, 5, 4)           \
-    FLOWMM_MB_MUL2(c12, c13, 6, 3, 2) FLOWMM_MB_MUL2(c14, c15, 7, 1, 0)                                         \
+// WIN = 16 x block number and MASK = 0xFFFFFFF0 held in a register, as asm operand references (the tag-insertion takes
+// one immediate only: with the mask as a literal too, each tag would first be moved into a register)
+#define FLOWMM_MB_STEP(c0, c1, c2, c3, c4, c5, c6, c7, c8, c9, c10, c11, c12, c13, c14, c15, WIN, MASK)         \
+    FLOWMM_MB_MUL2(c0, c1, 0, 15, 14, MASK) FLOWMM_MB_MUL2(c2, c3, 1, 13, 12, MASK) FLOWMM_MB_MUL2(c4, c5, 2, 11, 10, MASK) \
+    FLOWMM_MB_MUL2(c6, c7, 3, 9, 8, MASK) FLOWMM_MB_MUL2(c8, c9, 4, 7, 6, MASK) FLOWMM_MB_MUL2(c10, c11, 5, 5, 4, MASK)     \
+    FLOWMM_MB_MUL2(c12, c13, 6, 3, 2, MASK) FLOWMM_MB_MUL2(c14, c15, 7, 1, 0, MASK)                             \
     "max.f32 m0, a" #c0 ", a" #c1 ", a" #c2 ";\n\t"                                                             \
     "max.f32 m1, a" #c3 ", a" #c4 ", a" #c5 ";\n\t"                                                             \
     "max.f32 m2, a" #c6 ", a" #c7 ", a" #c8 ";\n\t"                                                             \
@@ -233,7 +234,7 @@ __device__ __forceinline__ MatchItem match_plan(const MatchTcArgs &A, int item) 
     "max.f32 m0, m0, m1, m2;\n\t"                                                                               \
     "max.f32 m3, m3, m4, a" #c15 ";\n\t"                                                                        \
     "max.f32 q0, m0, m3;\n\t"                                                                                   \
-    "and.b32 qm, q0, 0xFFFFFFF0;\n\t"                                                                           \
+    "and.b32 qm, q0, " MASK ";\n\t"                                                                             \
     "setp.gt.f32 p0, qm, %0;\n\t"                                                                               \
     "@p0 mov.b32 %0, qm;\n\t"                                                                                   \
     "@p0 lop3.b32 %1, q0, 15, " WIN ", 0xEA;\n\t"
@@ -251,10 +252,10 @@ __device__ __forceinline__ void match_block16(uint32_t taddr, uint32_t scales, f
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {a0, a1, a2, a3, a4, a5, a6, a7, a8, a9, a10, a11, a12, a13, a14, a15}, [%2];\n\t"
         FLOWMM_MB_LDS(0)
         "tcgen05.wait::ld.sync.aligned;\n\t"
-        FLOWMM_MB_STEP(0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, "%4")
+        FLOWMM_MB_STEP(0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, "%4", "%5")
         "}"
         : "+f"(best), "+r"(win)
-        : "r"(taddr), "r"(scales), "n"(16 * kBlk)
+        : "r"(taddr), "r"(scales), "n"(16 * kBlk), "r"(0xFFFFFFF0u)
         : "memory");
 }
 
@@ -266,12 +267,12 @@ __device__ __forceinline__ void match_block32(uint32_t taddr, uint32_t scales, f
         "a16, a17, a18, a19, a20, a21, a22, a23, a24, a25, a26, a27, a28, a29, a30, a31}, [%2];\n\t"
         FLOWMM_MB_LDS(0)
         "tcgen05.wait::ld.sync.aligned;\n\t"
-        FLOWMM_MB_STEP(0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, "%4")
+        FLOWMM_MB_STEP(0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, "%4", "%6")
         FLOWMM_MB_LDS(64)
-        FLOWMM_MB_STEP(16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, "%5")
+        FLOWMM_MB_STEP(16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, "%5", "%6")
         "}"
         : "+f"(best), "+r"(win)
-        : "r"(taddr), "r"(scales), "n"(16 * kBlk), "n"(16 * kBlk + 16)
+        : "r"(taddr), "r"(scales), "n"(16 * kBlk), "n"(16 * kBlk + 16), "r"(0xFFFFFFF0u)
         : "memory");
 }
 #undef FLOWMM_MB_MUL2
@@ -433,11 +434,13 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     } else {
                         const int nb = min(n_blocks - b0, kPer);     // blocks of this warp in this tile (may be <= 0)
                         // block before which the text group's winner is set aside (>= nb: not in this tile)
+                        // (splitting a ragged last tile evenly between the row's two warps was measured and is no faster:
+                        // the tile's arithmetic, not the longer of its two shares, is what takes the time)
                         const int pk = parked ? kPer : max(0, (p.t0 - (col0 + b0 * 16)) >> 4);
-                        const uint32_t sc = scale4 + b0 * 64;
+                        const uint32_t sc = scale4 + b0 * 64, tl = t_lane;
                         before = best;
                         if (nb == kPer && pk >= kPer) {
-                            match_blocks<kPer>(t_lane, sc, best, win);
+                            match_blocks<kPer>(tl, sc, best, win);
                         } else {
                             // (the group boundary is a multiple of 32 columns, the warp's share starts at one: pairs of blocks)
 #pragma unroll
@@ -446,10 +449,10 @@ match_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                                     if (i == pk) park(t);
                                     const bool two = i + 1 < nb;
                                     switch (i) {                     // (the block's number is a compile-time constant)
-                                        case 0: if (two) match_block32<0>(t_lane, sc, best, win); else match_block16<0>(t_lane, sc, best, win); break;
-                                        case 2: if (two) match_block32<2>(t_lane + 32, sc + 128, best, win); else match_block16<2>(t_lane + 32, sc + 128, best, win); break;
-                                        case 4: if (two) match_block32<4>(t_lane + 64, sc + 256, best, win); else match_block16<4>(t_lane + 64, sc + 256, best, win); break;
-                                        default: if (two) match_block32<6>(t_lane + 96, sc + 384, best, win); else match_block16<6>(t_lane + 96, sc + 384, best, win); break;
+                                        case 0: if (two) match_block32<0>(tl, sc, best, win); else match_block16<0>(tl, sc, best, win); break;
+                                        case 2: if (two) match_block32<2>(tl + 32, sc + 128, best, win); else match_block16<2>(tl + 32, sc + 128, best, win); break;
+                                        case 4: if (two) match_block32<4>(tl + 64, sc + 256, best, win); else match_block16<4>(tl + 64, sc + 256, best, win); break;
+                                        default: if (two) match_block32<6>(tl + 96, sc + 384, best, win); else match_block16<6>(tl + 96, sc + 384, best, win); break;
                                     }
                                 }
                             }
