@@ -97,8 +97,8 @@ void layout_merge(Layout &y, const flowmm_params &p, Take take) {
     const size_t UH = (size_t)p.n_units * p.n_kv_heads, B = p.n_keep, E = (size_t)p.seq_len - B, D = p.head_dim;
     y.max_pieces = (int)(B + E / kPiece + 1);
     y.max_parts = (int)(2 * (E / kPiece) + 2);
-    y.csr_passes = 1;
-    while (y.csr_passes < 4 && (B >> (8 * y.csr_passes)) != 0) ++y.csr_passes;
+    y.csr_passes = 1;                                        // digits of kCsrBits bits over the keys 0 .. B
+    while (y.csr_passes < 6 && (B >> (kCsrBits * y.csr_passes)) != 0) ++y.csr_passes;
     y.sort_a = take(UH * E * 4);
     y.sort_b = take(UH * E * 4);
     y.mem_tok = take(UH * E * 4);
@@ -580,8 +580,19 @@ flowmm_status run_merge(const flowmm_params &p, const Layout &y, const void *k, 
         c.off = at<int>(ws, y.off); c.piece_off = at<int>(ws, y.piece_off); c.part_off = at<int>(ws, y.part_off);
         c.piece_desc = at<int4>(ws, y.piece_desc); c.ticket = at<unsigned>(ws, y.ticket); c.slot_done = at<int>(ws, y.slot_done);
         c.B = p.n_keep; c.E = E; c.n_pass = y.csr_passes; c.max_pieces = y.max_pieces; c.merge_mode = p.merge_mode;
-        if (E <= 4096) build_csr_kernel<8><<<UH, 256, 0, st>>>(c);
-        else build_csr_kernel<32><<<UH, 1024, 0, st>>>(c);
+        // positions and keys as 16-bit arrays in shared memory when they fit (6 bytes per non-pivot), else through global memory
+        const size_t csr_smem = 6 * (((size_t)E + 7) & ~(size_t)7);
+        const bool staged = E < 65536 && p.n_keep < 65535 && csr_smem <= 200 * 1024;
+        if (staged) {
+            if (E <= 4096) {
+                if (cudaFuncSetAttribute(build_csr_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csr_smem) != cudaSuccess) return FLOWMM_ERR_CUDA;
+                build_csr_kernel<8, true><<<UH, 256, csr_smem, st>>>(c);
+            } else {
+                if (cudaFuncSetAttribute(build_csr_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csr_smem) != cudaSuccess) return FLOWMM_ERR_CUDA;
+                build_csr_kernel<32, true><<<UH, 1024, csr_smem, st>>>(c);
+            }
+        } else if (E <= 4096) build_csr_kernel<8, false><<<UH, 256, 0, st>>>(c);
+        else build_csr_kernel<32, false><<<UH, 1024, 0, st>>>(c);
         FLOWMM_LAUNCHED("build_csr");
         m.mem_tok = c.mem_tok; m.mem_w = c.mem_w; m.piece_desc = c.piece_desc;
         m.piece_off = c.piece_off; m.part_off = c.part_off; m.ticket = c.ticket; m.slot_done = c.slot_done;

@@ -1,5 +1,6 @@
 // Pivot selection (top-B per KV head) and the merge / compaction stage.
 #pragma once
+#include <type_traits>
 #include "common.cuh"
 
 namespace flowmm {
@@ -147,71 +148,120 @@ struct CsrArgs {
 
 __device__ __forceinline__ int csr_key(int m, int B) { return m < 0 ? B : m; }   // dropped tokens sort last
 
-// grid = U*Hkv, block = 32 * NW threads (warp w owns a contiguous range of the input).
-template <int NW>
+constexpr int kCsrBits = 6, kCsrBins = 1 << kCsrBits;      // digit width of the sort
+
+// Lanes of the warp that hold the same digit as this one, among the valid lanes: a vote per bit and as many logic
+// operations (the match instruction gives the same set, but its unit is slow and shared by the SM's warps).
+__device__ __forceinline__ uint32_t digit_peers(int digit, bool valid) {
+    uint32_t mine = __ballot_sync(0xFFFFFFFFu, valid);
+#pragma unroll
+    for (int b = 0; b < kCsrBits; ++b) {
+        const uint32_t vote = __ballot_sync(0xFFFFFFFFu, (digit >> b) & 1);
+        mine &= ((digit >> b) & 1) ? vote : ~vote;
+    }
+    return mine;
+}
+
+// grid = U*Hkv, block = 32 * NW threads (warp w owns a contiguous range of the input).  n_pass passes of kCsrBits bits.
+// The sort gathers keys by position and scatters positions, 4 or 2 bytes at a time, which an SM's global-memory path
+// takes at about one access per clock: with kStaged (E and B below 65536 and 6 E bytes of dynamic shared memory) the
+// keys and both position buffers are 16-bit arrays in shared memory and only the results touch global memory.
+template <int NW, bool kStaged>
 __global__ void __launch_bounds__(32 * NW) build_csr_kernel(const CsrArgs A) {
     constexpr int kThreads = 32 * NW;
-    __shared__ int counters[NW][257];               // [warp][digit], padded
+    constexpr int kBatch = 8;                       // steps of 32 positions whose loads are in flight together
+    using Pos = std::conditional_t<kStaged, uint16_t, int>;
+    extern __shared__ __align__(16) uint16_t csr_smem[];   // kStaged: keys[Ep], positions[2][Ep], Ep = E rounded up to 8
+    __shared__ int counters[NW][kCsrBins + 1];      // [warp][digit], padded
     __shared__ int scratch[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int uh = blockIdx.x;
     if (uh == 0 && tid == 0) *A.ticket = 0u;
     const int *match = A.match + (int64_t)uh * A.E;
-    int *bufs[2] = {A.sort_a + (int64_t)uh * A.E, A.sort_b + (int64_t)uh * A.E};
+    const int Ep = (A.E + 7) & ~7;
+    Pos *bufs[2];
+    if constexpr (kStaged) {
+        // (the buffer that holds the final order comes last: keys and the other buffer are then one free region of 4 Ep bytes)
+        const int fin = (A.n_pass - 1) & 1;
+        bufs[fin] = csr_smem + 2 * Ep; bufs[fin ^ 1] = csr_smem + Ep;
+        for (int i = tid; i < A.E; i += kThreads) csr_smem[i] = (uint16_t)csr_key(match[i], A.B);
+        __syncthreads();
+    } else {
+        bufs[0] = A.sort_a + (int64_t)uh * A.E; bufs[1] = A.sort_b + (int64_t)uh * A.E;
+    }
+    auto key_of = [&](int j) -> int {
+        if constexpr (kStaged) return csr_smem[j]; else return csr_key(match[j], A.B);
+    };
     const int per_warp = ((A.E + NW - 1) / NW + 31) / 32 * 32;     // multiple of 32
     const int lo = warp * per_warp, hi = min(A.E, lo + per_warp);
+    const int end = min(lo + per_warp, ((hi + 31) / 32) * 32);
 
     for (int pass = 0; pass < A.n_pass; ++pass) {
-        const int shift = 8 * pass;
-        const int *src = pass == 0 ? nullptr : bufs[(pass - 1) & 1];
-        int *dst = bufs[pass & 1];
-        for (int i = tid; i < NW * 257; i += kThreads) (&counters[0][0])[i] = 0;
-        __syncthreads();
-        // count digits, warp-private counters
-        for (int t = lo; t < lo + per_warp && t < ((hi + 31) / 32) * 32; t += 32) {
-            const int idx = t + lane;
-            const bool valid = idx < hi;
-            const int j = valid ? (src ? src[idx] : idx) : 0;
-            const int digit = valid ? (csr_key(match[j], A.B) >> shift) & 255 : 256 + lane;
-            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-            if (valid && lane == __ffs(peers) - 1) counters[warp][digit] += __popc(peers);
-            __syncwarp();
-        }
-        __syncthreads();
-        // exclusive scan in (digit, warp) order: thread t covers 8 consecutive entries
-        int vals[8], sum = 0;
+        const int shift = kCsrBits * pass;
+        const Pos *src = pass == 0 ? nullptr : bufs[(pass - 1) & 1];
+        Pos *dst = bufs[pass & 1];
+        // The positions and their keys are fetched kBatch steps at a time (the loads of a step depend on each other,
+        // those of different steps do not); a step past the warp's range has no valid lane and changes nothing.
+        auto fetch = [&](int t0, int (&jv)[kBatch], int (&dg)[kBatch]) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int idx = tid * 8 + e;            // idx = digit * NW + warp
-            vals[e] = counters[idx % NW][idx / NW];
-            sum += vals[e];
-        }
-        int total;
-        int run = block_exclusive_scan(sum, scratch, total);
+            for (int b = 0; b < kBatch; ++b) {
+                const int idx = t0 + 32 * b + lane;
+                jv[b] = idx < hi ? (src ? (int)src[idx] : idx) : -1;
+            }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int idx = tid * 8 + e;
-            counters[idx % NW][idx / NW] = run;
-            run += vals[e];
+            for (int b = 0; b < kBatch; ++b) dg[b] = jv[b] >= 0 ? (key_of(jv[b]) >> shift) & (kCsrBins - 1) : 0;
+        };
+        // count the warp's positions by digit (order does not matter here: shared-memory atomics on the warp's own counters)
+        for (int d = lane; d < kCsrBins; d += 32) counters[warp][d] = 0;
+        __syncwarp();
+        for (int t0 = lo; t0 < end; t0 += 32 * kBatch) {
+            int jv[kBatch], dg[kBatch];
+            fetch(t0, jv, dg);
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b)
+                if (jv[b] >= 0) atomicAdd(&counters[warp][dg[b]], 1);
         }
         __syncthreads();
-        // scatter, in order inside each warp's range
-        for (int t = lo; t < lo + per_warp && t < ((hi + 31) / 32) * 32; t += 32) {
-            const int idx = t + lane;
-            const bool valid = idx < hi;
-            const int j = valid ? (src ? src[idx] : idx) : 0;
-            const int digit = valid ? (csr_key(match[j], A.B) >> shift) & 255 : 256 + lane;
-            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-            const int rank = __popc(peers & lanemask_lt());
-            if (valid) dst[counters[warp][digit] + rank] = j;
-            __syncwarp();
-            if (valid && lane == __ffs(peers) - 1) counters[warp][digit] += __popc(peers);
-            __syncwarp();
+        // exclusive scan in (digit, warp) order: thread t holds the kPerThread consecutive entries from kPerThread t on,
+        // entry e being digit = e / NW, warp = e % NW
+        {
+            constexpr int kPerThread = kCsrBins / 32;
+            int vals[kPerThread], sum = 0;
+#pragma unroll
+            for (int e = 0; e < kPerThread; ++e) {
+                const int idx = tid * kPerThread + e;
+                vals[e] = counters[idx % NW][idx / NW];
+                sum += vals[e];
+            }
+            int total;
+            int run = block_exclusive_scan(sum, scratch, total);
+            __syncthreads();
+#pragma unroll
+            for (int e = 0; e < kPerThread; ++e) {
+                const int idx = tid * kPerThread + e;
+                counters[idx % NW][idx / NW] = run;
+                run += vals[e];
+            }
+        }
+        __syncthreads();
+        // scatter, in order inside each warp's range: the warp's counters now hold the next free place of each digit
+        for (int t0 = lo; t0 < end; t0 += 32 * kBatch) {
+            int jv[kBatch], dg[kBatch];
+            fetch(t0, jv, dg);
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const bool valid = jv[b] >= 0;
+                const uint32_t mine = digit_peers(dg[b], valid);
+                if (valid) dst[counters[warp][dg[b]] + __popc(mine & lanemask_lt())] = (Pos)jv[b];
+                __syncwarp();
+                if (valid && lane == __ffs(mine) - 1) counters[warp][dg[b]] += __popc(mine);
+                __syncwarp();
+            }
         }
         __syncthreads();
         __threadfence_block();
     }
-    const int *sorted = bufs[(A.n_pass - 1) & 1];
+    const Pos *sorted = bufs[(A.n_pass - 1) & 1];
     int *off = A.off + (int64_t)uh * (A.B + 1);
     int *piece_off = A.piece_off + (int64_t)uh * (A.B + 1);
     int *part_off = A.part_off + (int64_t)uh * (A.B + 1);
@@ -221,20 +271,38 @@ __global__ void __launch_bounds__(32 * NW) build_csr_kernel(const CsrArgs A) {
         const float *sim = A.match_sim + (int64_t)uh * A.E;
         int *mem_tok = A.mem_tok + (int64_t)uh * A.E;
         float *mem_w = A.mem_w + (int64_t)uh * A.E;
+        // ... and off[s] = number of sorted entries with key < s: entry i starts every slot above its predecessor's
+        // key up to its own, the last entry also ends the slots above its key (E > 0: the kernel is not launched otherwise)
         for (int i = tid; i < A.E; i += kThreads) {
             const int j = sorted[i];
-            mem_tok[i] = evi[j];
-            mem_w[i] = A.merge_mode == 1 ? 1.f : __expf(sim[j] - 1.f);
+            const int key = key_of(j);
+            const int prev = i > 0 ? key_of(sorted[i - 1]) : -1;
+            if constexpr (!kStaged) {
+                mem_tok[i] = evi[j];
+                mem_w[i] = A.merge_mode == 1 ? 1.f : __expf(sim[j] - 1.f);
+            }
+            for (int s2 = prev + 1; s2 <= key; ++s2) off[s2] = i;
+            if (i == A.E - 1)
+                for (int s2 = key + 1; s2 <= A.B; ++s2) off[s2] = A.E;
         }
-    }
-    // off[s] = number of sorted entries with key < s (binary search on the sorted order)
-    for (int s = tid; s <= A.B; s += kThreads) {
-        int a = 0, b = A.E;
-        while (a < b) {
-            const int mid = (a + b) >> 1;
-            if (csr_key(match[sorted[mid]], A.B) < s) a = mid + 1; else b = mid;
+        if constexpr (kStaged) {
+            // the gathers by position go through shared memory as well: the token positions, then the similarities, are
+            // copied in order into the region the keys and the spare buffer have left, and picked from there
+            int *stage_i = reinterpret_cast<int *>(csr_smem);
+            float *stage_f = reinterpret_cast<float *>(csr_smem);
+            __syncthreads();                                     // the keys are not read any more
+            for (int i = tid; i < A.E; i += kThreads) stage_i[i] = evi[i];
+            __syncthreads();
+            for (int i = tid; i < A.E; i += kThreads) mem_tok[i] = stage_i[sorted[i]];
+            __syncthreads();
+            if (A.merge_mode == 1) {
+                for (int i = tid; i < A.E; i += kThreads) mem_w[i] = 1.f;
+            } else {
+                for (int i = tid; i < A.E; i += kThreads) stage_f[i] = sim[i];
+                __syncthreads();
+                for (int i = tid; i < A.E; i += kThreads) mem_w[i] = __expf(stage_f[sorted[i]] - 1.f);
+            }
         }
-        off[s] = a;
     }
     __syncthreads();
     // pieces per slot and partial records per slot, exclusive scans over the slots
