@@ -67,9 +67,31 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int i = tid; i < 256; i += nthreads) hist[i] = 0;
         __syncthreads();
-        for (int i = tid; i < L; i += nthreads) {
-            const uint32_t key = select_key(imp[i], i >= first_forced);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        // Eight keys per thread are in flight at a time, and a thread adds runs of equal digits at once: the first
+        // digits (sign and exponent) are nearly the same for all keys, which would put every thread's every add on one counter.
+        {
+            int run_bin = -1, run_cnt = 0;
+            for (int base = 0; base < L; base += 8 * nthreads) {
+                uint32_t keys[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int i = base + e * nthreads + tid;
+                    keys[e] = i < L ? select_key(imp[i], i >= first_forced) : 0u;
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int i = base + e * nthreads + tid;
+                    if (i < L && (keys[e] & mask) == prefix) {
+                        const int bin = (keys[e] >> shift) & 255;
+                        if (bin != run_bin) {
+                            if (run_cnt > 0) atomicAdd(&hist[run_bin], run_cnt);
+                            run_bin = bin; run_cnt = 0;
+                        }
+                        ++run_cnt;
+                    }
+                }
+            }
+            if (run_cnt > 0) atomicAdd(&hist[run_bin], run_cnt);
         }
         __syncthreads();
         if (tid < 32) {                              // walk down from the largest digit, 8 digits per lane
@@ -99,21 +121,36 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
         mask |= 0xFFu << shift;
     }
     // keys > prefix are all kept; of the keys == prefix the first `need` (by position) are kept
+    // (four consecutive positions per thread and round: a quarter of the block-wide scans)
     int eq_seen = 0, kept_seen = 0;
-    for (int base = 0; base < L; base += nthreads) {
-        const int i = base + tid;
-        uint32_t key = 0;
-        bool valid = i < L;
-        if (valid) key = select_key(imp[i], i >= first_forced);
-        const int is_eq = valid && key == prefix;
+    for (int base = 0; base < L; base += 4 * nthreads) {
+        const int i0 = base + 4 * tid;
+        uint32_t key[4];
+        int n_eq = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            key[e] = i0 + e < L ? select_key(imp[i0 + e], i0 + e >= first_forced) : 0u;
+            n_eq += i0 + e < L && key[e] == prefix;
+        }
         int total_eq;
-        const int eq_rank = eq_seen + block_exclusive_scan(is_eq, scratch, total_eq);
-        const int keep = valid && (key > prefix || (is_eq && eq_rank < need));
+        int eq_rank = eq_seen + block_exclusive_scan(n_eq, scratch, total_eq);
+        int keep[4], n_keep = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const bool valid = i0 + e < L, is_eq = valid && key[e] == prefix;
+            keep[e] = valid && (key[e] > prefix || (is_eq && eq_rank < need));
+            eq_rank += is_eq;
+            n_keep += keep[e];
+        }
         int total_keep;
-        const int pos = kept_seen + block_exclusive_scan(keep, scratch, total_keep);
-        if (valid) {
-            if (keep) ret[pos] = i;
-            else evi[i - pos] = i;
+        int pos = kept_seen + block_exclusive_scan(n_keep, scratch, total_keep);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (i0 + e < L) {
+                if (keep[e]) ret[pos] = i0 + e;
+                else evi[i0 + e - pos] = i0 + e;
+            }
+            pos += keep[e];
         }
         eq_seen += total_eq;
         kept_seen += total_keep;
