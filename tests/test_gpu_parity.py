@@ -77,6 +77,14 @@ def test_ragged_shapes(dtype, D):
         _random_case(rng, U, Hq, Hkv, D, L, W, B, dtype, tau=3.0, tau_mode=O.TAU_REL, theta=0.5)
 
 
+def test_member_lists_too_long_for_the_shared_memory_sort():
+    # 35 700 non-pivots per head: six bytes each no longer fit the sort's shared-memory staging, so the member lists of the
+    # staged merge are sorted through global memory (the shorter lists of every other case take the staged sort)
+    rng = np.random.default_rng(4242)
+    stats = _random_case(rng, 1, 2, 1, 128, 36000, 16, 300, F.BF16, vis_frac=0.8, tau=3.0, tau_mode=O.TAU_REL, theta=0.5)
+    assert stats["kv_rows_checked"] == stats["kv_rows_total"]
+
+
 def test_short_context_kernel_boundaries():
     """Shapes around the switch points of the one-pass scoring kernel (32 proxy rows per KV head, up to 8 key
     tiles), the short-list matching kernel (up to 256 candidate columns, i.e. B <= 224) and the tensor-core merge
