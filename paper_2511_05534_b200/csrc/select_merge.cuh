@@ -121,7 +121,7 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
         mask |= 0xFFu << shift;
     }
     // keys > prefix are all kept; of the keys == prefix the first `need` (by position) are kept
-    // (four consecutive positions per thread and round: a quarter of the block-wide scans)
+    // (four consecutive positions per thread and iteration: a quarter of the block-wide scans)
     int eq_seen = 0, kept_seen = 0;
     for (int base = 0; base < L; base += 4 * nthreads) {
         const int i0 = base + 4 * tid;
