@@ -403,17 +403,38 @@ flowmm_status run_layer_flow(const flowmm_params &p, const float *cross_mass, fl
     return FLOWMM_OK;
 }
 
+// What the preparation of the tensor-core matching step needs (candidate layout per head; see match_tc.cuh).
+MatchPrepArgs match_prep_args(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
+                              const uint8_t *mod, const int32_t *retained, const int32_t *evicted, void *ws) {
+    MatchPrepArgs g;
+    g.k = k; g.importance = importance; g.modality = mod;
+    g.retained = retained; g.evicted = evicted;
+    g.cand_k = at<__nv_bfloat16>(ws, y.cand_k); g.cand_scale = at<float>(ws, y.cand_scale);
+    g.cand_slot = at<int>(ws, y.cand_slot); g.cand_count = at<int>(ws, y.cand_count);
+    g.rank = at<int>(ws, y.rank); g.tile_mod = at<uint8_t>(ws, y.tile_mod);
+    g.Hkv = p.n_kv_heads; g.L = p.seq_len; g.B = p.n_keep; g.E = p.seq_len - p.n_keep; g.Ctot = y.c_tot; g.n_rt = y.n_rt;
+    g.tau_eff = tau_effective(p);
+    for (int i = 0; i < 3; ++i) g.ks[i] = p.k_stride[i];
+    g.copy_here = y.c_tot <= 256;
+    g.status = at<int>(ws, y.status);
+    return g;
+}
+
 // cross_mass != nullptr: the launch also applies Eq. 6 and the theta rule to the final masses (rho may be nullptr)
+// prep != nullptr: each block goes on to prepare its head's matching candidates (the fused call, tensor-core matching)
 flowmm_status run_select(const flowmm_params &p, const float *importance, int32_t *retained, int32_t *evicted,
                          cudaStream_t st, float *cross_mass = nullptr, float *rho = nullptr,
-                         int32_t *strategy = nullptr, const float *cross_part = nullptr, int n_parts = 0) {
+                         int32_t *strategy = nullptr, const float *cross_part = nullptr, int n_parts = 0,
+                         const MatchPrepArgs *prep = nullptr) {
     const int few = p.n_units * p.n_kv_heads < 2 * tc::sm_count();       // few heads: more threads per head
     const int threads = few ? (p.seq_len <= 512 ? 256 : kSelectThreads) : p.seq_len <= 2048 ? 256 : p.seq_len <= 8192 ? 512 : kSelectThreads;
     SelectFlow f;
     f.cross_part = cross_part; f.n_parts = n_parts; f.cross_mass = cross_mass; f.rho = rho; f.strategy = strategy; f.Hq = p.n_q_heads; f.Hkv = p.n_kv_heads;
     f.theta = p.theta; f.flow_mode = p.flow_mode;
+    MatchPrepArgs none = {};
     select_topb_kernel<<<p.n_units * p.n_kv_heads, threads, 0, st>>>(importance, p.seq_len, p.n_keep, p.window,
-                                                                           p.keep_window, retained, evicted, f);
+                                                                           p.keep_window, retained, evicted, f,
+                                                                           prep ? *prep : none, prep ? 1 : 0);
     FLOWMM_LAUNCHED("select_topb");
     return FLOWMM_OK;
 }
@@ -422,23 +443,15 @@ flowmm_status run_select(const flowmm_params &p, const float *importance, int32_
 flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
                            const uint8_t *mod, const int32_t *retained, const int32_t *evicted,
                            const int32_t *strategy, int32_t *match, float *match_sim, void *ws, cudaStream_t st,
-                           int2 *tokmap) {
+                           int2 *tokmap, bool prepared) {
     const int UH = p.n_units * p.n_kv_heads, E = p.seq_len - p.n_keep;
-    MatchPrepArgs g;
-    g.k = k; g.importance = importance; g.modality = mod;
-    g.retained = retained; g.evicted = evicted;
-    g.cand_k = at<__nv_bfloat16>(ws, y.cand_k); g.cand_scale = at<float>(ws, y.cand_scale);
-    g.cand_slot = at<int>(ws, y.cand_slot); g.cand_count = at<int>(ws, y.cand_count);
-    g.rank = at<int>(ws, y.rank); g.tile_mod = at<uint8_t>(ws, y.tile_mod);
-    g.Hkv = p.n_kv_heads; g.L = p.seq_len; g.B = p.n_keep; g.E = E; g.Ctot = y.c_tot; g.n_rt = y.n_rt;
-    g.tau_eff = tau_effective(p);
-    for (int i = 0; i < 3; ++i) g.ks[i] = p.k_stride[i];
-    g.copy_here = y.c_tot <= 256;
-    g.status = at<int>(ws, y.status);
-    // few heads: a head's lists are walked by more threads, the GPU is not full either way
-    const int prep_threads = UH >= 4 * tc::sm_count() ? 256 : UH >= 2 * tc::sm_count() ? 512 : 1024;
-    match_prepare_kernel<<<UH, prep_threads, 0, st>>>(g);
-    FLOWMM_LAUNCHED("match_prepare");
+    const MatchPrepArgs g = match_prep_args(p, y, k, importance, mod, retained, evicted, ws);
+    if (!prepared) {                                 // (the fused call's selection launch has done it already)
+        // few heads: a head's lists are walked by more threads, the GPU is not full either way
+        const int prep_threads = UH >= 4 * tc::sm_count() ? 256 : UH >= 2 * tc::sm_count() ? 512 : 1024;
+        match_prepare_kernel<<<UH, prep_threads, 0, st>>>(g);
+        FLOWMM_LAUNCHED("match_prepare");
+    }
     if (!g.copy_here) {
         match_gather_kernel<<<dim3(UH, (y.c_tot + 63) / 64), 256, 0, st>>>(g);
         FLOWMM_LAUNCHED("match_gather");
@@ -493,10 +506,11 @@ flowmm_status run_match_tc(const flowmm_params &p, const Layout &y, const void *
 // tokmap != nullptr (only with the short-list tensor-core kernel): also write the tensor-core merge's table
 flowmm_status run_match(const flowmm_params &p, const Layout &y, const void *k, const float *importance,
                         const uint8_t *mod, const int32_t *retained, const int32_t *evicted, const int32_t *strategy,
-                        int32_t *match, float *match_sim, void *ws, cudaStream_t st, int2 *tokmap = nullptr) {
+                        int32_t *match, float *match_sim, void *ws, cudaStream_t st, int2 *tokmap = nullptr,
+                        bool prepared = false) {
     const int E = p.seq_len - p.n_keep;
     if (E == 0) return FLOWMM_OK;
-    if (use_tc(p)) return run_match_tc(p, y, k, importance, mod, retained, evicted, strategy, match, match_sim, ws, st, tokmap);
+    if (use_tc(p)) return run_match_tc(p, y, k, importance, mod, retained, evicted, strategy, match, match_sim, ws, st, tokmap, prepared);
     float *rn = at<float>(ws, y.rn);
     const int64_t rows = (int64_t)p.n_units * p.n_kv_heads * p.seq_len;
     const int lanes = p.head_dim / (p.dtype == FLOWMM_BF16 ? 8 : 4);
@@ -729,12 +743,15 @@ flowmm_status flowmm_compress_layer(const flowmm_params *p, const void *q_win, c
     int n_parts = 0;
     FLOWMM_TRY(run_score(*p, y, q_win, k, modality, importance, cross_mass, ws, st, &n_parts));
     // Eq. 6 and the theta rule ride along with the selection launch (which first adds up the partial masses, if any)
+    // ... and so does the candidate layout of the tensor-core matching step
+    const bool prep_in_select = p->seq_len > p->n_keep && use_tc(*p);
+    const MatchPrepArgs prep = match_prep_args(*p, y, k, importance, modality, retained_idx, evicted_idx, ws);
     FLOWMM_TRY(run_select(*p, importance, retained_idx, evicted_idx, st, cross_mass, rho, strategy,
-                          n_parts > 0 ? at<float>(ws, y.cross_part) : nullptr, n_parts));
+                          n_parts > 0 ? at<float>(ws, y.cross_part) : nullptr, n_parts, prep_in_select ? &prep : nullptr));
     // when both the short-list matching kernel and the tensor-core merge apply, the former writes the latter's table
     const bool map_in_match = p->seq_len > p->n_keep && use_tc(*p) && y.c_tot <= mst::kMaxCols && merge_is_tc(*p);
     FLOWMM_TRY(run_match(*p, y, k, importance, modality, retained_idx, evicted_idx, strategy, match, match_sim, ws, st,
-                         map_in_match ? at<int2>(ws, y.tokmap) : nullptr));
+                         map_in_match ? at<int2>(ws, y.tokmap) : nullptr, prep_in_select));
     FLOWMM_TRY(run_merge(*p, y, k, v, retained_idx, evicted_idx, match, match_sim, k_out, v_out, ws, st, map_in_match));
     return FLOWMM_OK;
 }

@@ -65,11 +65,11 @@ __device__ __forceinline__ void match_gather_rows(const MatchPrepArgs &A, int uh
     }
 }
 
-// grid = U*Hkv, block = 256 to 1024 (a multiple of 32).
-__global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs A) {
-    __shared__ int scratch[33];
-    __shared__ int s_ntext;
-    const int tid = threadIdx.x, uh = blockIdx.x, u = uh / A.Hkv, h = uh % A.Hkv;
+// The preparation of one (unit, head) by its whole block (256 to 1024 threads, a multiple of 32); `scratch` = 33 ints
+// and `s_ntext` = one int of shared memory.  Also called at the end of the selection kernel, which has just written
+// this head's index lists.
+__device__ __forceinline__ void match_prepare_head(const MatchPrepArgs &A, int uh, int *scratch, int *s_ntext) {
+    const int tid = threadIdx.x, u = uh / A.Hkv, h = uh % A.Hkv;
     const int *ret = A.retained + (int64_t)uh * A.B;
     const int *evi = A.evicted + (int64_t)uh * A.E;
     const float *imp = A.importance + (int64_t)uh * A.L;
@@ -99,9 +99,9 @@ __global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs
     }
     int total;
     block_exclusive_scan(n_text, scratch, total);
-    if (tid == 0) s_ntext = total;
+    if (tid == 0) *s_ntext = total;
     __syncthreads();
-    const int t0 = (s_ntext + 31) & ~31;
+    const int t0 = (*s_ntext + 31) & ~31;
     int seen_t = 0, seen_v = 0;
     for (int base = 0; base < A.B; base += blockDim.x) {
         const int s = base + tid;
@@ -123,6 +123,13 @@ __global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs
     if (tid == 0) { A.cand_count[2 * uh] = seen_t; A.cand_count[2 * uh + 1] = seen_v; }
     __syncthreads();
     if (A.copy_here) match_gather_rows(A, uh, 0, A.Ctot, tid, blockDim.x);
+}
+
+// grid = U*Hkv, block = 256 to 1024 (a multiple of 32).
+__global__ void __launch_bounds__(1024) match_prepare_kernel(const MatchPrepArgs A) {
+    __shared__ int scratch[33];
+    __shared__ int s_ntext;
+    match_prepare_head(A, blockIdx.x, scratch, &s_ntext);
 }
 
 // The gather step of the preparation as a kernel of its own for long candidate lists, so that many

@@ -2,6 +2,7 @@
 #pragma once
 #include <type_traits>
 #include "common.cuh"
+#include "match_tc.cuh"
 
 namespace flowmm {
 
@@ -31,9 +32,11 @@ struct SelectFlow {
     int flow_mode;
 };
 
+// with_prepare: the block goes on to lay out the head's matching candidates (match_prepare_head) from the lists it has
+// just written, which saves the short-context workloads a launch and a second pass over the same few kilobytes.
 __global__ void __launch_bounds__(kSelectThreads)
 select_topb_kernel(const float *importance, int L, int B, int W, int keep_window, int *retained, int *evicted,
-                   const SelectFlow F) {
+                   const SelectFlow F, const MatchPrepArgs P, int with_prepare) {
     __shared__ int hist[256];
     __shared__ int scratch[33];
     __shared__ uint32_t s_prefix;
@@ -154,6 +157,10 @@ select_topb_kernel(const float *importance, int L, int B, int W, int keep_window
         }
         eq_seen += total_eq;
         kept_seen += total_keep;
+    }
+    if (with_prepare) {
+        __syncthreads();                                 // this block's lists are complete and visible to all its threads
+        match_prepare_head(P, blockIdx.x, scratch, &s_need);
     }
 }
 
